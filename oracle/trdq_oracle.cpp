@@ -1,0 +1,293 @@
+// CPU oracle for the time-rotated quantized linear layer (TR-DQ).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what the
+// hot path computes, written from the paper's definitions.  It shares no code,
+// header, table or helper with the CUDA library, and the library never calls it.
+// Only the tests, the smoke check and the benchmark's cpu-baseline leg use it.
+//
+// What is followed, step by step (names as in the paper):
+//   * Sec. 3.1, Eq. 1-2: uniform integer quantizer with nearest rounding, used in
+//     its symmetric signed 8-bit form (zero-point 0, scale = absmax / 127);
+//     per-token scales for activations and per-output-channel scales for weights
+//     ("per-token quantization for activations and per-channel ... for weights").
+//   * Sec. 3.1, Eq. 4: channel scaling vector Delta.  Following Eq. 10 the online
+//     side MULTIPLIES X by Delta_t and the offline side multiplies W by 1/Delta_t.
+//   * Sec. 3.2, Eq. 8: block-diagonal orthogonal rotation, blocks of 2^n x 2^n;
+//     here n = 7 and every block is diag(d) * H_128 / sqrt(128) with H_128 the
+//     Sylvester-Walsh-Hadamard matrix and d a +-1 vector per time-step group.
+//   * Sec. 3.2, Eq. 10: F_t(X, W) = G_t(X) . H_t(W) with the parameter set chosen
+//     by the current time-step; "dynamic quantization ... calculating quantization
+//     parameters online" for the activations.
+//
+// Parity notes.  The quantizer, the integer GEMM and the dequantising epilogue are
+// pinned by the tests against closed forms and brute force.  Two things are
+// conventions of this build that the paper does not fix ("parity unpinned" by the
+// paper): the order of the fp32 additions inside the butterfly (h = 1, 2, ..., 64,
+// natural output order) and the 4-bit weight storage format (two's complement
+// nibbles, even k in the low nibble, one fp32 scale per 128 consecutive k).
+//
+// Build: g++ -O2 -ffp-contract=off -fopenmp -shared -fPIC (no fast-math).
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+constexpr int kBlock = 128;
+// 2^-3.5 = 1/sqrt(128): the normalisation that makes H_128/sqrt(128) orthogonal.
+constexpr double kHadamardNorm = 0.08838834764831845;
+
+inline float bf16_to_float(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+// In-place Walsh-Hadamard butterfly on 128 fp32 values, unnormalised.
+// Stage h pairs index i with i+h (bit h of i clear): (a, b) -> (a + b, a - b).
+// Natural (Sylvester) order: out[i] = sum_j (-1)^popcount(i & j) in[j].
+void butterfly128(float* u) {
+  for (int h = 1; h < kBlock; h <<= 1) {
+    for (int i = 0; i < kBlock; ++i) {
+      if ((i & h) == 0) {
+        const float a = u[i];
+        const float b = u[i + h];
+        u[i] = a + b;
+        u[i + h] = a - b;
+      }
+    }
+  }
+}
+
+// Scale one row by the fused vector and rotate every 128-block (Eq. 10, G_t / H_t).
+void rotate_row(const uint16_t* row_bf16, const float* vec, int K, float* out) {
+  for (int c = 0; c < K; c += kBlock) {
+    float u[kBlock];
+    for (int i = 0; i < kBlock; ++i) u[i] = bf16_to_float(row_bf16[c + i]) * vec[c + i];
+    butterfly128(u);
+    for (int i = 0; i < kBlock; ++i) out[c + i] = u[i];
+  }
+}
+
+// Symmetric signed quantizer over `n` values with `qmax` levels each side (Eq. 1-2, z = 0).
+// Returns the scale; writes integer codes.
+float quantize_span(const float* v, int n, float qmax, int8_t* q) {
+  float amax = 0.0f;
+  for (int i = 0; i < n; ++i) amax = std::fmax(amax, std::fabs(v[i]));
+  const float scale = amax / qmax;
+  const float inv = amax > 0.0f ? qmax / amax : 0.0f;
+  const int lim = static_cast<int>(qmax);
+  for (int i = 0; i < n; ++i) {
+    const float scaled = v[i] * inv;
+    int r = static_cast<int>(std::nearbyintf(scaled));  // default mode: ties to even
+    if (r > lim) r = lim;
+    if (r < -lim) r = -lim;
+    q[i] = static_cast<int8_t>(r);
+  }
+  return scale;
+}
+
+}  // namespace
+
+extern "C" {
+
+// Time-step -> group (Sec. 3.2: the parameter set is selected by the current
+// time-step).  Returns g with bounds[g] <= t < bounds[g+1], or -1.
+int oracle_group_of(const int32_t* bounds, int num_groups, int t) {
+  for (int g = 0; g < num_groups; ++g)
+    if (bounds[g] <= t && t < bounds[g + 1]) return g;
+  return -1;
+}
+
+// Fused per-channel vectors of one group, computed in double and rounded once:
+//   act[j]    = fl32(d[j] * Delta[j] * 2^-3.5)   (applied to X, Eq. 10 G_t)
+//   weight[j] = fl32(d[j] / Delta[j] * 2^-3.5)   (applied to W, Eq. 10 H_t)
+// smooth == nullptr means Delta = 1.
+void oracle_fused_vectors(const int8_t* signs, const float* smooth, int K, float* act, float* weight) {
+  for (int j = 0; j < K; ++j) {
+    const double d = static_cast<double>(signs[j]);
+    const double delta = smooth ? static_cast<double>(smooth[j]) : 1.0;
+    act[j] = static_cast<float>(d * delta * kHadamardNorm);
+    weight[j] = static_cast<float>(d / delta * kHadamardNorm);
+  }
+}
+
+// Rotated rows in fp32 (no quantisation): v = (x o vec) . BlockDiag(H_128).
+void oracle_rotate(const uint16_t* x_bf16, int64_t ldx, int M, int K, const float* vec, float* v) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) rotate_row(x_bf16 + static_cast<int64_t>(m) * ldx, vec, K, v + static_cast<int64_t>(m) * K);
+}
+
+// Per-row symmetric int8 quantiser on already-rotated fp32 rows.
+void oracle_quantize_rows(const float* v, int M, int K, int8_t* codes, float* scales) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    scales[m] = quantize_span(v + static_cast<int64_t>(m) * K, K, 127.0f, codes + static_cast<int64_t>(m) * K);
+}
+
+// Online activation path: rotate then quantise per token.
+void oracle_rotate_quantize(const uint16_t* x_bf16, int64_t ldx, int M, int K, const float* act_vec,
+                            int8_t* codes, float* scales) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) {
+    std::vector<float> v(K);
+    rotate_row(x_bf16 + static_cast<int64_t>(m) * ldx, act_vec, K, v.data());
+    scales[m] = quantize_span(v.data(), K, 127.0f, codes + static_cast<int64_t>(m) * K);
+  }
+}
+
+// Offline weight path, 8-bit: rotate each output channel's row with the weight
+// vector, quantise per output channel.
+void oracle_prepare_w8(const uint16_t* w_bf16, int N, int K, const float* weight_vec, int8_t* codes, float* scales) {
+  oracle_rotate_quantize(w_bf16, K, N, K, weight_vec, codes, scales);
+}
+
+// Offline weight path, 4-bit: one scale per (output channel, 128 consecutive k),
+// codes in [-7, 7], two per byte (even k in the low nibble, two's complement).
+void oracle_prepare_w4(const uint16_t* w_bf16, int N, int K, const float* weight_vec, uint8_t* packed, float* scales) {
+  const int groups = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n) {
+    std::vector<float> v(K);
+    rotate_row(w_bf16 + static_cast<int64_t>(n) * K, weight_vec, K, v.data());
+    for (int kg = 0; kg < groups; ++kg) {
+      int8_t q[kBlock];
+      scales[static_cast<int64_t>(n) * groups + kg] = quantize_span(v.data() + kg * kBlock, kBlock, 7.0f, q);
+      for (int i = 0; i < kBlock; i += 2) {
+        const uint8_t lo = static_cast<uint8_t>(q[i]) & 0xF;
+        const uint8_t hi = static_cast<uint8_t>(q[i + 1]) & 0xF;
+        packed[(static_cast<int64_t>(n) * K + kg * kBlock + i) / 2] = static_cast<uint8_t>(lo | (hi << 4));
+      }
+    }
+  }
+}
+
+// Sign-extending unpack of the 4-bit storage format back to int8 codes [N, K].
+void oracle_unpack_w4(const uint8_t* packed, int64_t count, int8_t* codes) {
+  for (int64_t i = 0; i < count; ++i) {
+    const uint8_t byte = packed[i / 2];
+    const int nib = (i & 1) ? (byte >> 4) : (byte & 0xF);
+    codes[i] = static_cast<int8_t>(nib >= 8 ? nib - 16 : nib);
+  }
+}
+
+// Integer GEMM (Eq. 10: G_t(X) . H_t(W) on the integer codes): exact int32 sums.
+void oracle_gemm_i32(const int8_t* q, const int8_t* qw, int M, int N, int K, int32_t* acc) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      int32_t s = 0;
+      for (int k = 0; k < K; ++k)
+        s += static_cast<int32_t>(q[static_cast<int64_t>(m) * K + k]) * static_cast<int32_t>(qw[static_cast<int64_t>(n) * K + k]);
+      acc[static_cast<int64_t>(m) * N + n] = s;
+    }
+}
+
+// Dequantising epilogue: y = acc * sx[m] * sw[n] + bias[n], evaluated in double and
+// rounded once to fp32.  bias may be null.
+void oracle_epilogue(const int32_t* acc, const float* sx, const float* sw, const uint16_t* bias_bf16, int M, int N, float* y) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      double r = static_cast<double>(acc[static_cast<int64_t>(m) * N + n]) * static_cast<double>(sx[m]) * static_cast<double>(sw[n]);
+      if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      y[static_cast<int64_t>(m) * N + n] = static_cast<float>(r);
+    }
+}
+
+// W8A8 linear on a row subset: rows[i] selects the token; y is [num_rows, N].
+void oracle_linear_w8_rows(const int8_t* q, const float* sx, const int8_t* qw, const float* sw, const uint16_t* bias_bf16,
+                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+#pragma omp parallel for schedule(static)
+  for (int i = 0; i < num_rows; ++i) {
+    const int64_t m = rows[i];
+    for (int n = 0; n < N; ++n) {
+      int32_t s = 0;
+      for (int k = 0; k < K; ++k)
+        s += static_cast<int32_t>(q[m * K + k]) * static_cast<int32_t>(qw[static_cast<int64_t>(n) * K + k]);
+      double r = static_cast<double>(s) * static_cast<double>(sx[m]) * static_cast<double>(sw[n]);
+      if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      y[static_cast<int64_t>(i) * N + n] = static_cast<float>(r);
+    }
+  }
+}
+
+// W4A8 linear on a row subset.  Every 128-wide k group has its own exact int32
+// partial sum, scaled by that group's weight scale:
+//   y = sx[m] * sum_kg (acc_kg * sw4[n, kg]) + bias[n]     (double, rounded once)
+void oracle_linear_w4_rows(const int8_t* q, const float* sx, const uint8_t* packed, const float* sw4, const uint16_t* bias_bf16,
+                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+  const int groups = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int i = 0; i < num_rows; ++i) {
+    const int64_t m = rows[i];
+    for (int n = 0; n < N; ++n) {
+      double total = 0.0;
+      for (int kg = 0; kg < groups; ++kg) {
+        int32_t s = 0;
+        for (int k = kg * kBlock; k < (kg + 1) * kBlock; ++k) {
+          const uint8_t byte = packed[(static_cast<int64_t>(n) * K + k) / 2];
+          const int nib = (k & 1) ? (byte >> 4) : (byte & 0xF);
+          const int wq = nib >= 8 ? nib - 16 : nib;
+          s += static_cast<int32_t>(q[m * K + k]) * wq;
+        }
+        total += static_cast<double>(s) * static_cast<double>(sw4[static_cast<int64_t>(n) * groups + kg]);
+      }
+      double r = static_cast<double>(sx[m]) * total;
+      if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      y[static_cast<int64_t>(i) * N + n] = static_cast<float>(r);
+    }
+  }
+}
+
+// ---- fp64 cross-check path (structurally different from the butterfly) -------
+// Dense K x K rotation of one group, R = diag(d) . BlockDiag(H_128) / sqrt(128),
+// with H built by the Sylvester recursion H_2n = [[H, H], [H, -H]].
+void oracle_dense_rotation(const int8_t* signs, int K, double* R) {
+  std::vector<double> H(kBlock * kBlock, 0.0);
+  H[0] = 1.0;
+  for (int n = 1; n < kBlock; n <<= 1)
+    for (int i = 0; i < n; ++i)
+      for (int j = 0; j < n; ++j) {
+        const double h = H[i * kBlock + j];
+        H[i * kBlock + (j + n)] = h;
+        H[(i + n) * kBlock + j] = h;
+        H[(i + n) * kBlock + (j + n)] = -h;
+      }
+  const double norm = 1.0 / std::sqrt(static_cast<double>(kBlock));
+  for (int64_t i = 0; i < static_cast<int64_t>(K) * K; ++i) R[i] = 0.0;
+  for (int c = 0; c < K; c += kBlock)
+    for (int i = 0; i < kBlock; ++i)
+      for (int j = 0; j < kBlock; ++j)
+        R[static_cast<int64_t>(c + i) * K + (c + j)] = static_cast<double>(signs[c + i]) * H[i * kBlock + j] * norm;
+}
+
+// C[M,N] = A[M,K] . B[K,N], plain triple loop in double.
+void oracle_matmul_f64(const double* A, const double* B, int M, int K, int N, double* C) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      double s = 0.0;
+      for (int k = 0; k < K; ++k) s += A[static_cast<int64_t>(m) * K + k] * B[static_cast<int64_t>(k) * N + n];
+      C[static_cast<int64_t>(m) * N + n] = s;
+    }
+}
+
+int oracle_num_threads() {
+  int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+  {
+#pragma omp single
+    n = omp_get_num_threads();
+  }
+#endif
+  return n;
+}
+
+}  // extern "C"

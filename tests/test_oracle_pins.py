@@ -1,0 +1,376 @@
+"""Pins for the CPU oracle: every check compares it with something other than itself
+(a textbook definition, a closed form, an invariant the paper states, a library
+routine it does not use, or brute force on tiny inputs)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import trdq_oracle as O
+from paper_2503_06564_b200 import workloads as WL
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+C_NORM = 2.0 ** -3.5
+
+
+def bf16(x):
+    return WL.to_bf16_bits(np.asarray(x, dtype=np.float64))
+
+
+def f32_of(bits):
+    return WL.bf16_bits_to_f32(bits)
+
+
+def unit_vectors(K=128):
+    return bf16(np.eye(K))
+
+
+def identity_vec_smooth():
+    """smooth value that makes the fused *activation* vector exactly +-1.0f."""
+    return np.float32(2.0 ** 3.5)
+
+
+# --------------------------------------------------------------------------- #
+# rotation (Eq. 8, Eq. 10)
+# --------------------------------------------------------------------------- #
+def test_fused_vectors_values():
+    rng = np.random.default_rng(1)
+    K = 256
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    a, b = O.fused_vectors(signs, None)
+    # Delta = 1: both vectors are d * 2^-3.5 rounded to fp32
+    assert np.array_equal(a, b)
+    assert np.array_equal(np.sign(a).astype(np.int8), signs)
+    assert np.allclose(a.astype(np.float64) ** 2 * 128.0, 1.0, rtol=2e-7)
+    smooth = rng.uniform(0.05, 20.0, K).astype(np.float32)
+    a, b = O.fused_vectors(signs, smooth)
+    # act carries Delta, weight carries 1/Delta: a*b = 1/128, a/b = Delta^2
+    assert np.allclose(a.astype(np.float64) * b.astype(np.float64) * 128.0, 1.0, rtol=3e-7)
+    assert np.allclose(a.astype(np.float64) / b.astype(np.float64), smooth.astype(np.float64) ** 2, rtol=3e-7)
+    assert np.array_equal(np.sign(a).astype(np.int8), signs)
+    assert np.array_equal(np.sign(b).astype(np.int8), signs)
+
+
+def test_unit_act_vector_trick():
+    signs = np.ones(128, np.int8)
+    a, _ = O.fused_vectors(signs, np.full(128, identity_vec_smooth(), np.float32))
+    assert np.all(a == np.float32(1.0))
+    _, b = O.fused_vectors(signs, np.full(128, np.float32(2.0 ** -3.5), np.float32))
+    assert np.all(b == np.float32(1.0))
+
+
+def test_butterfly_is_sylvester_natural_order():
+    """Row j of the transform of the identity is (-1)^popcount(i & j): natural order, no bit reversal."""
+    ones = np.ones(128, np.float32)
+    v = O.rotate(unit_vectors(), ones)          # v[j, i] = H[j][i]
+    i = np.arange(128)
+    pop = np.array([[bin(a & b).count("1") for a in i] for b in i])
+    assert np.array_equal(v, ((-1.0) ** pop).astype(np.float32))
+    golden = np.loadtxt(os.path.join(GOLDEN, "hadamard8_sylvester.txt"))
+    assert np.array_equal(v[:8, :8], golden.astype(np.float32))
+
+
+def test_butterfly_closed_forms():
+    ones = np.ones(128, np.float32)
+    x = np.zeros((3, 128))
+    x[0, 0] = 3.0            # H(alpha e0) = alpha * ones
+    x[1, :] = 1.0            # H(ones) = 128 e0
+    x[2, 5] = -2.0
+    v = O.rotate(bf16(x), ones)
+    assert np.array_equal(v[0], np.full(128, 3.0, np.float32))
+    e0 = np.zeros(128, np.float32); e0[0] = 128.0
+    assert np.array_equal(v[1], e0)
+    # involution: H(H(x)) = 128 x  (values stay small integers => exact in bf16/fp32)
+    rng = np.random.default_rng(7)
+    xi = rng.integers(-1, 2, size=(4, 128)).astype(np.float64)
+    once = O.rotate(bf16(xi), ones)
+    assert np.all(np.abs(once) <= 128)
+    twice = O.rotate(bf16(once.astype(np.float64) / 128.0), ones)   # /128 exact; bf16 holds k/128, |k|<=128
+    assert np.array_equal(twice, xi.astype(np.float32))
+
+
+def test_dense_rotation_is_orthogonal():
+    rng = np.random.default_rng(3)
+    K = 384
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    R = O.dense_rotation(signs)
+    assert np.max(np.abs(R @ R.T - np.eye(K))) < 1e-6
+    assert np.max(np.abs(R.T @ R - np.eye(K))) < 1e-6
+    # block-diagonal: nothing outside the 128 x 128 diagonal blocks
+    mask = np.kron(np.eye(K // 128), np.ones((128, 128))) > 0
+    assert np.all(R[~mask] == 0.0)
+    assert np.allclose(np.abs(R[mask]), C_NORM)
+
+
+def test_computational_invariance_fp64():
+    """(X Delta R)(R^T Delta^-1 W) = X W  (Eq. 9 / Eq. 10) in double to 1e-10."""
+    rng = np.random.default_rng(4)
+    M, K, N = 8, 256, 24
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    delta = rng.uniform(0.1, 8.0, K)
+    X = rng.standard_normal((M, K))
+    W = rng.standard_normal((K, N))            # paper orientation: C_in x C_out
+    R = O.dense_rotation(signs)
+    G = O.matmul_f64(X * delta[None, :], R)
+    H = O.matmul_f64(np.ascontiguousarray(R.T), W / delta[:, None])
+    Y = O.matmul_f64(G, H)
+    ref = X @ W
+    assert np.max(np.abs(Y - ref)) / np.max(np.abs(ref)) < 1e-10
+
+
+def test_butterfly_matches_dense_fp64_product():
+    """fp32 butterfly vs. the fp64 dense product, within the fp32 summation bound."""
+    rng = np.random.default_rng(5)
+    M, K = 16, 384
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.2, 5.0, K).astype(np.float32)
+    xb = bf16(rng.standard_normal((M, K)) * 3.0)
+    a, b = O.fused_vectors(signs, smooth)
+    v = O.rotate(xb, a).astype(np.float64)
+    x = f32_of(xb).astype(np.float64)
+    R = O.dense_rotation(signs)
+    dense = (x * smooth.astype(np.float64)[None, :]) @ R
+    # bound: 8 roundings along each path, each relative 2^-24, on sum_j |x_j a_j|
+    mag = np.abs(x * a.astype(np.float64)[None, :]).reshape(M, K // 128, 128).sum(axis=2)
+    bound = np.repeat(mag, 128, axis=1) * 128 * 2.0 ** -24 + 1e-12
+    assert np.all(np.abs(v - dense) <= bound)
+    assert np.max(np.abs(v - dense)) > 0      # the two paths are really different computations
+    # weight side uses 1/Delta
+    vw = O.rotate(xb, b).astype(np.float64)
+    dense_w = (x / smooth.astype(np.float64)[None, :]) @ R
+    assert np.all(np.abs(vw - dense_w) <= np.repeat(
+        np.abs(x * b.astype(np.float64)[None, :]).reshape(M, K // 128, 128).sum(axis=2), 128, axis=1) * 128 * 2.0 ** -24 + 1e-12)
+
+
+def test_block_diagonal_locality():
+    rng = np.random.default_rng(6)
+    K = 512
+    a, _ = O.fused_vectors(np.ones(K, np.int8), None)
+    x = rng.standard_normal((1, K))
+    x2 = x.copy()
+    x2[0, 128 + 17] += 5.0
+    v1 = O.rotate(bf16(x), a)
+    v2 = O.rotate(bf16(x2), a)
+    changed = np.nonzero(v1[0] != v2[0])[0]
+    assert changed.min() >= 128 and changed.max() < 256 and changed.size == 128
+
+
+# --------------------------------------------------------------------------- #
+# quantizer (Eq. 1-2, symmetric signed form; per token)
+# --------------------------------------------------------------------------- #
+def test_quantizer_error_bound_and_extremes():
+    rng = np.random.default_rng(8)
+    v = (rng.standard_normal((64, 256)) * rng.uniform(0.01, 100.0, (64, 1))).astype(np.float32)
+    q, s = O.quantize_rows(v)
+    assert q.dtype == np.int8 and s.shape == (64,)
+    amax = np.abs(v).max(axis=1)
+    assert np.allclose(s.astype(np.float64) * 127.0, amax.astype(np.float64), rtol=1e-6)
+    err = np.abs(v.astype(np.float64) - s.astype(np.float64)[:, None] * q.astype(np.float64))
+    assert np.all(err <= s.astype(np.float64)[:, None] * (0.5 + 1e-5))
+    assert q.min() >= -127 and q.max() <= 127
+    rows = np.arange(64)
+    arg = np.abs(v).argmax(axis=1)
+    assert np.all(np.abs(q[rows, arg]) == 127)
+    assert np.array_equal(np.sign(q[rows, arg]), np.sign(v[rows, arg]).astype(np.int8))
+
+
+def test_quantizer_zero_row_and_row_independence():
+    rng = np.random.default_rng(9)
+    v = rng.standard_normal((5, 128)).astype(np.float32)
+    v[2] = 0.0
+    q, s = O.quantize_rows(v)
+    assert s[2] == 0.0 and np.all(q[2] == 0)
+    # dynamic per-token scale: a row's result does not depend on the other rows
+    perm = np.array([4, 0, 3, 1, 2])
+    q2, s2 = O.quantize_rows(v[perm])
+    assert np.array_equal(q2, q[perm]) and np.array_equal(s2, s[perm])
+    v3 = v.copy(); v3[0] *= 1000.0
+    q3, s3 = O.quantize_rows(v3)
+    assert np.array_equal(q3[1:], q[1:]) and np.array_equal(s3[1:], s[1:])
+
+
+def test_quantizer_round_half_to_even():
+    table = np.loadtxt(os.path.join(GOLDEN, "rounding_ties.txt"))
+    vals, expect = table[:, 0], table[:, 1].astype(np.int64)
+    for p in (-3, 0, 5):
+        row = np.zeros(128, np.float32)
+        row[0] = 127.0 * 2.0 ** p           # absmax => inverse scale is exactly 2^-p
+        row[1:1 + vals.size] = (vals * 2.0 ** p).astype(np.float32)
+        q, s = O.quantize_rows(row[None, :])
+        assert s[0] == np.float32(2.0 ** p)
+        assert q[0, 0] == 127
+        assert np.array_equal(q[0, 1:1 + vals.size].astype(np.int64), expect)
+
+
+def test_rotate_quantize_equals_its_two_steps():
+    rng = np.random.default_rng(10)
+    xb = bf16(rng.standard_normal((9, 256)))
+    a, _ = O.fused_vectors((rng.integers(0, 2, 256) * 2 - 1).astype(np.int8), None)
+    q, s = O.rotate_quantize(xb, a)
+    q2, s2 = O.quantize_rows(O.rotate(xb, a))
+    assert np.array_equal(q, q2) and np.array_equal(s, s2)
+
+
+# --------------------------------------------------------------------------- #
+# integer GEMM and epilogue (Eq. 10)
+# --------------------------------------------------------------------------- #
+def test_int_gemm_brute_force_and_numpy():
+    q = np.array([[1, -2, 3, 4], [127, 127, -127, 0]], np.int8)
+    w = np.array([[1, 1, 1, 1], [0, -1, 2, -3], [127, 127, -127, 5]], np.int8)
+    acc = O.gemm_i32(q, w)
+    # written out by hand
+    assert acc.tolist() == [[6, -4, -488], [127, -381, 48387]]
+    rng = np.random.default_rng(11)
+    q = rng.integers(-127, 128, (37, 384), dtype=np.int8)
+    w = rng.integers(-127, 128, (29, 384), dtype=np.int8)
+    assert np.array_equal(O.gemm_i32(q, w).astype(np.int64), q.astype(np.int64) @ w.astype(np.int64).T)
+    # extreme magnitude stays exact in int32
+    q = np.full((1, 4096), 127, np.int8); w = np.full((1, 4096), -127, np.int8)
+    assert O.gemm_i32(q, w)[0, 0] == -4096 * 127 * 127
+
+
+def test_epilogue_special_cases():
+    rng = np.random.default_rng(12)
+    acc = rng.integers(-256, 257, (6, 10)).astype(np.int32)
+    ones_m, ones_n = np.ones(6, np.float32), np.ones(10, np.float32)
+    assert np.array_equal(O.epilogue(acc, ones_m, ones_n, None), acc.astype(np.float32))
+    bias = bf16(rng.standard_normal(10))
+    y = O.epilogue(np.zeros((6, 10), np.int32), ones_m, ones_n, bias)
+    assert np.array_equal(y, np.broadcast_to(f32_of(bias), (6, 10)))
+    # per-token scale acts on rows, per-channel scale on columns (powers of two: exact)
+    sx = np.array([1, 2, 4, 8, 16, 32], np.float32)
+    sw = (2.0 ** -np.arange(10)).astype(np.float32)
+    y = O.epilogue(acc, sx, sw, None)
+    assert np.array_equal(y, (acc * sx[:, None] * sw[None, :]).astype(np.float32))
+    y_rows = O.linear_w8_rows(np.eye(6, 128, dtype=np.int8), sx, np.ones((10, 128), np.int8), sw, None, np.array([5, 0]))
+    assert np.array_equal(y_rows, np.stack([32.0 * sw, 1.0 * sw]).astype(np.float32))
+
+
+def _w8a8(xb, wb, biasb, signs, smooth):
+    a, b = O.fused_vectors(signs, smooth)
+    q, sx = O.rotate_quantize(xb, a)
+    qw, sw = O.prepare_w8(wb, b)
+    return O.epilogue(O.gemm_i32(q, qw), sx, sw, biasb)
+
+
+def test_end_to_end_close_to_fp64_linear():
+    """The whole quantised path reproduces X W + bias up to quantisation noise (Eq. 10)."""
+    wl = WL.WORKLOADS[0]
+    li = WL.make_layer_inputs(wl, 0, M=32)
+    x = f32_of(li.x).astype(np.float64); w = f32_of(li.w).astype(np.float64)
+    ref = x @ w.T + f32_of(li.bias).astype(np.float64)[None, :]
+    rng = np.random.default_rng(13)
+    smooth = rng.uniform(0.5, 2.0, (1, li.layer.K)).astype(np.float32)
+    for sm in (None, smooth[0]):
+        y = _w8a8(li.x, li.w, li.bias, li.signs[0], sm).astype(np.float64)
+        rel = np.linalg.norm(y - ref) / np.linalg.norm(ref)
+        assert rel < 0.02, rel
+    rows = np.array([3, 31, 0])
+    a, b = O.fused_vectors(li.signs[1], None)
+    q, sx = O.rotate_quantize(li.x, a); qw, sw = O.prepare_w8(li.w, b)
+    full = O.epilogue(O.gemm_i32(q, qw), sx, sw, li.bias)
+    assert np.array_equal(O.linear_w8_rows(q, sx, qw, sw, li.bias, rows), full[rows])
+
+
+def test_rotation_reduces_outliers_and_error():
+    """Sec. 3.2: rotation spreads massive outliers, shrinking the per-token range and the W8A8 error."""
+    wl = WL.WORKLOADS[0]
+    li = WL.make_layer_inputs(wl, 0, M=64)
+    x = f32_of(li.x).astype(np.float64); w = f32_of(li.w).astype(np.float64)
+    a, b = O.fused_vectors(li.signs[0], None)
+    v = O.rotate(li.x, a)
+    before = np.abs(x).max(axis=1).mean()
+    after = np.abs(v).max(axis=1).mean()
+    assert before / after > 3.0
+    ref = x @ w.T
+    y_rot = O.epilogue(O.gemm_i32(*[t for t in (O.rotate_quantize(li.x, a)[0], O.prepare_w8(li.w, b)[0])]),
+                       O.rotate_quantize(li.x, a)[1], O.prepare_w8(li.w, b)[1], None)
+    qx, sx = O.quantize_rows(f32_of(li.x)); qw, sw = O.quantize_rows(f32_of(li.w))
+    y_plain = O.epilogue(O.gemm_i32(qx, qw), sx, sw, None)
+    e_rot = np.linalg.norm(y_rot - ref); e_plain = np.linalg.norm(y_plain - ref)
+    assert e_rot < 0.5 * e_plain
+
+
+# --------------------------------------------------------------------------- #
+# 4-bit weights
+# --------------------------------------------------------------------------- #
+def _w4_rows_for_pairs():
+    """Rows whose rotated values are the period-4 pattern (a, b, +-7, r): exact small numbers."""
+    pairs = [(a, b) for a in range(-7, 8) for b in range(-7, 8)]
+    idx = np.arange(128)
+    s = np.zeros((len(pairs), 128))
+    for r, (a, b) in enumerate(pairs):
+        s2 = (a - 7) / 2.0 if b <= a else (a + 7) / 2.0
+        s[r, 1] = (a - b) / 2.0
+        s[r, 2] = s2
+        s[r, 0] = (a + b) / 2.0 - s2
+    return pairs, s
+
+
+def test_w4_pack_exhaustive_nibble_pairs():
+    pairs, s = _w4_rows_for_pairs()
+    _, wvec = O.fused_vectors(np.ones(128, np.int8), np.full(128, np.float32(2.0 ** -3.5), np.float32))
+    assert np.all(wvec == np.float32(1.0))
+    sb = bf16(s)
+    assert np.array_equal(f32_of(sb).astype(np.float64), s)      # inputs are exact in bf16
+    v = O.rotate(sb, wvec)
+    packed, scales = O.prepare_w4(sb, wvec)
+    assert packed.shape == (len(pairs), 64) and scales.shape == (len(pairs), 1)
+    assert np.all(scales == np.float32(1.0))
+    for r, (a, b) in enumerate(pairs):
+        assert v[r, 0] == a and v[r, 1] == b and abs(v[r, 2]) == 7
+        assert packed[r, 0] == ((a & 0xF) | ((b & 0xF) << 4))
+        assert packed[r, 1] == ((int(v[r, 2]) & 0xF) | ((int(v[r, 3]) & 0xF) << 4))
+    assert np.array_equal(O.unpack_w4(packed).astype(np.float32), v)
+
+
+def test_w4_group_scales_and_linear():
+    rng = np.random.default_rng(14)
+    N, K, M = 12, 384, 7
+    wb = bf16(rng.standard_normal((N, K)) * 0.02)
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    a, b = O.fused_vectors(signs, None)
+    packed, sw4 = O.prepare_w4(wb, b)
+    v = O.rotate(wb, b).reshape(N, K // 128, 128)
+    amax = np.abs(v).max(axis=2)
+    assert np.allclose(sw4.astype(np.float64) * 7.0, amax.astype(np.float64), rtol=1e-6)
+    q4 = O.unpack_w4(packed).reshape(N, K // 128, 128)
+    assert q4.min() >= -7 and q4.max() <= 7
+    assert np.all(np.abs(v - sw4[:, :, None] * q4) <= sw4[:, :, None] * (0.5 + 1e-5))
+    # linear: sum over k-groups of exact int partials times the group scale
+    xb = bf16(rng.standard_normal((M, K)))
+    q, sx = O.rotate_quantize(xb, a)
+    bias = bf16(rng.standard_normal(N) * 0.01)
+    y = O.linear_w4_rows(q, sx, packed, sw4, bias, np.arange(M))
+    deq = (q4.astype(np.float64) * sw4.astype(np.float64)[:, :, None]).reshape(N, K)
+    ref = sx.astype(np.float64)[:, None] * (q.astype(np.float64) @ deq.T) + f32_of(bias).astype(np.float64)[None, :]
+    assert np.allclose(y, ref, rtol=1e-6, atol=1e-9)
+    x = f32_of(xb).astype(np.float64); w = f32_of(wb).astype(np.float64)
+    full = x @ w.T + f32_of(bias).astype(np.float64)[None, :]
+    assert np.linalg.norm(y - full) / np.linalg.norm(full) < 0.15
+
+
+# --------------------------------------------------------------------------- #
+# time-step groups (Sec. 3.2, Time-Rotation)
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5])
+def test_group_of_exhaustive(G):
+    bounds = WL.group_bounds(G)
+    assert bounds[0] == 0 and bounds[-1] == 1000 and np.all(np.diff(bounds) > 0)
+    t = np.arange(1000)
+    got = np.array([O.group_of(bounds, int(ti)) for ti in t])
+    assert np.array_equal(got, np.searchsorted(bounds, t, side="right") - 1)
+    assert O.group_of(bounds, -1) == -1 and O.group_of(bounds, 1000) == -1
+
+
+def test_time_step_selects_parameter_set():
+    wl = WL.WORKLOADS[0]
+    li = WL.make_layer_inputs(wl, 0, M=8)
+    codes = {}
+    for t in (0, 250, 499, 500, 750, 999):
+        g = O.group_of(li.t_bounds, t)
+        a, _ = O.fused_vectors(li.signs[g], None)
+        codes[t] = O.rotate_quantize(li.x, a)[0]
+    assert np.array_equal(codes[0], codes[250]) and np.array_equal(codes[250], codes[499])
+    assert np.array_equal(codes[500], codes[750]) and np.array_equal(codes[750], codes[999])
+    assert not np.array_equal(codes[499], codes[500])
