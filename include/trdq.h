@@ -1,0 +1,161 @@
+/* trdq.h -- C ABI of the time-rotated quantized linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the online path of TR-DQ's rotated quantized linear layer
+ * (Sec. 3.2, Eq. 10):
+ *
+ *     F_t(X, W) = G_t(X) . H_t(W),   G_t(X) = (X . Delta_t) . R_t,   H_t(W) = R_t^T . (Delta_t^-1 . W)
+ *
+ * with the parameter set {R_t, Delta_t} chosen by the current diffusion time-step t
+ * ("Time-Rotation"), activations quantized dynamically per token and weights per
+ * output channel (Sec. 3.1, Eq. 1-2, used in symmetric signed form: zero-point 0,
+ * scale = absmax / qmax, nearest rounding with ties to even).
+ *
+ * The rotation R_g of a time-step group g is block diagonal (Eq. 8) with blocks of
+ * 128 x 128: R_g = diag(d_g) . BlockDiag(H_128) / sqrt(128), H_128 the Sylvester
+ * Walsh-Hadamard matrix in natural order and d_g a +-1 vector.  The per-group channel
+ * scaling Delta_g (Eq. 4-5; the per-time-step hyper-parameter alpha of Eq. 5 enters
+ * through it) multiplies X online and divides W offline, exactly as Eq. 10 is written.
+ *
+ * Conventions
+ *   - Every matrix is row major with the reduction dimension K (= C_in) contiguous:
+ *     X [M, K], W [N, K] (the transpose of the paper's C_in x C_out matrix), Y [M, N].
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host
+ *     memory.  bf16 tensors are passed as `const void*` / `void*` to 2-byte elements.
+ *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = the legacy default stream).
+ *   - All device work is enqueued asynchronously on `stream`; no entry point
+ *     synchronises unless its comment says so.  The online calls (trdq_rotate_quantize,
+ *     trdq_linear, trdq_linear_cfg, trdq_gemm_i32) allocate no memory.
+ *   - The caller owns every tensor it passes.  The library owns only the opaque
+ *     trdq_rotation / trdq_weights objects until their _destroy call.
+ *   - Errors are reported by return code only; the library never aborts, traps or
+ *     prints.  Argument errors are found on the host before anything is launched.
+ *     NaN/Inf in X or W give unspecified codes (not checked).
+ *   - There is no CPU fallback: without a CUDA device every call that needs one
+ *     returns TRDQ_ERR_CUDA.
+ */
+#ifndef TRDQ_H_
+#define TRDQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TRDQ_BLOCK 128        /* rotation block size 2^n (Eq. 8), n = 7 */
+#define TRDQ_MAX_K 131072     /* keeps |sum_k q*qw| <= K*127*127 below 2^31 */
+
+typedef enum trdq_status {
+  TRDQ_OK = 0,
+  TRDQ_ERR_NULL = 1,      /* a required pointer is NULL */
+  TRDQ_ERR_SHAPE = 2,     /* K % 128 != 0, N % 16 != 0, M < 0, K > TRDQ_MAX_K, block != 128, ld too small */
+  TRDQ_ERR_ALIGN = 3,     /* a device pointer or row stride is not 16-byte aligned */
+  TRDQ_ERR_TIMESTEP = 4,  /* t outside [t_bounds[0], t_bounds[G]) */
+  TRDQ_ERR_GROUP = 5,     /* num_groups < 1, bounds not strictly ascending, sign not +-1, smooth <= 0 */
+  TRDQ_ERR_WBITS = 6,     /* wbits is neither 8 nor 4, or the call does not support this weight format */
+  TRDQ_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (no device, launch error, ...) */
+  TRDQ_ERR_NOMEM = 8,     /* host or device allocation failed */
+  TRDQ_ERR_TIMEOUT = 9,   /* a bounded device-side wait expired (see trdq_device_status) */
+  TRDQ_ERR_MISMATCH = 10  /* objects passed together were built for different K / groups */
+} trdq_status;
+
+/* Description of the per-group transforms (Time-Rotation, Sec. 3.2).  All arrays are
+ * host memory and are copied by trdq_rotation_create. */
+typedef struct trdq_rotation_spec {
+  int32_t K;                /* C_in; multiple of 128 */
+  int32_t block;            /* rotation block size; must be 128 */
+  int32_t num_groups;       /* G >= 1 time-step groups */
+  const int32_t* t_bounds;  /* host [G+1], strictly ascending; group g covers t_bounds[g] <= t < t_bounds[g+1] */
+  const int8_t* signs;      /* host [G][K], each +1 or -1: the diagonal d_g */
+  const float* smooth;      /* host [G][K], > 0: Delta_g as multiplied onto X (Eq. 10); NULL = all ones */
+} trdq_rotation_spec;
+
+typedef struct trdq_rotation trdq_rotation; /* per-group device tables of one C_in */
+typedef struct trdq_weights trdq_weights;   /* H_t(W) of one linear layer, quantized, for all groups */
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* trdq_status_string(trdq_status s);
+
+/* Builds the per-group tables.  For each group the two fused fp32 vectors
+ *   act[j]    = fl32(d[j] * Delta[j] * 2^-3.5)     (applied to X)
+ *   weight[j] = fl32(d[j] / Delta[j] * 2^-3.5)     (applied to W)
+ * are formed in double precision, rounded once and uploaded (2^-3.5 = 1/sqrt(128) is the
+ * Hadamard normalisation).  Synchronous (blocking copies).  `*out` is set only on TRDQ_OK. */
+trdq_status trdq_rotation_create(const trdq_rotation_spec* spec, trdq_rotation** out);
+trdq_status trdq_rotation_destroy(trdq_rotation* rot);
+
+/* Time-step -> group (Sec. 3.2: the parameter set is selected by the current time-step).
+ * Pure host arithmetic.  TRDQ_ERR_TIMESTEP if t is outside the covered range. */
+trdq_status trdq_group_of(const trdq_rotation* rot, int32_t t, int32_t* g);
+
+/* The same lookup on a bare table (host [num_groups+1], strictly ascending), for callers that
+ * schedule sampling steps before any device object exists.  Pure host arithmetic. */
+trdq_status trdq_find_group(const int32_t* t_bounds, int32_t num_groups, int32_t t, int32_t* g);
+
+/* Offline side of Eq. 10: for every group g, rotate each output channel's row of W with
+ * the weight vector of g (H_t(W) = R_t^T Delta_t^-1 W, written on rows of W^T) and quantize
+ *   wbits = 8: per output channel, codes int8 [N, K] in [-127, 127], scale fp32 [N] = absmax / 127;
+ *   wbits = 4: per (output channel, 128 consecutive k), codes in [-7, 7] packed two per byte
+ *              (uint8 [N, K/2], even k in the low nibble, two's complement), scale fp32 [N, K/128] = absmax / 7.
+ * W_bf16: dev [N, K] contiguous, 16-byte aligned.  N % 16 == 0.  Allocates the G quantized copies
+ * (cudaMalloc) and enqueues the kernels on `stream`; the object may be used on the same stream
+ * right away.  `*out` is set only on TRDQ_OK. */
+trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, int32_t N, int32_t wbits,
+                                 trdq_weights** out, void* stream);
+trdq_status trdq_weights_destroy(trdq_weights* w);
+
+/* Shape and format of a prepared layer (any output pointer may be NULL). */
+trdq_status trdq_weights_info(const trdq_weights* w, int32_t* N, int32_t* K, int32_t* wbits, int32_t* num_groups);
+
+/* Device pointers to group g's quantized codes and scales (layouts as in trdq_prepare_weights);
+ * the memory stays owned by `w`. */
+trdq_status trdq_weights_view(const trdq_weights* w, int32_t g, const void** Wq, const float** scales);
+
+/* Online activation path G_t(X) followed by dynamic per-token quantization (Sec. 3.1 Eq. 1-2,
+ * Sec. 3.2 "calculating quantization parameters online"):
+ *   v[m, :]   = (x[m, :] o act_g) . BlockDiag(H_128), fp32 butterflies in the order h = 1, 2, ..., 64
+ *   scales[m] = absmax_k |v[m, k]| / 127
+ *   codes[m,k]= rne(v[m, k] * fl32(127 / absmax))     (all-zero row: scale 0, codes 0)
+ * with g the group of time-step t.  X_bf16: dev [M, ldx] (ldx >= K elements, ldx % 8 == 0, base
+ * 16-byte aligned); codes: dev int8 [M, K] contiguous, 16-byte aligned; scales: dev fp32 [M].
+ * M == 0 is a no-op.  Both CFG halves are simply rows of the same call. */
+trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M,
+                                 int8_t* codes, float* scales, void* stream);
+
+/* Integer GEMM of Eq. 10 on the codes with the dequantizing epilogue:
+ *   wbits = 8:  y[m, n] = bf16( (sum_k q[m,k] * qw_g[n,k]) * sx[m] * sw_g[n] + bias[n] )
+ *   wbits = 4:  y[m, n] = bf16( sx[m] * sum_kg sw4_g[n,kg] * (sum_{k in kg} q[m,k] * qw4_g[n,k]) + bias[n] )
+ * int8 x int8 (int4) products accumulate exactly in int32 on the tensor cores; the epilogue runs in
+ * fp32.  codes: dev int8 [M, K] contiguous, 16-byte aligned; scales: dev fp32 [M]; bias_bf16: dev [N]
+ * or NULL; Y_bf16: dev [M, ldy], ldy >= N, ldy % 8 == 0, base 16-byte aligned.  Conditional and
+ * unconditional CFG rows stacked in one call share a single read of the weights. */
+trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
+                        const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
+
+/* Same as trdq_linear for two separately stored row segments (the conditional and the
+ * unconditional CFG half) of the same time-step, in ONE launch so that each weight tile is
+ * fetched once for both.  Segment s has M[s] rows (either may be 0). */
+trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
+                            const int32_t M[2], const void* bias_bf16, void* const Y_bf16[2], const int64_t ldy[2],
+                            void* stream);
+
+/* Raw accumulators of the integer GEMM (wbits = 8 only): acc[m, n] = sum_k q[m,k] * qw_g[n,k],
+ * dev int32 [M, ldacc], ldacc >= N, ldacc % 4 == 0.  Exists so that the exact integer result
+ * can be checked bit for bit. */
+trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes, int32_t M, int32_t* acc, int64_t ldacc,
+                          void* stream);
+
+/* Reads and clears the device-side status word of the current device.  Kernels never spin
+ * without bound: a wait on a memory barrier that exceeds its limit sets a bit in this word
+ * and the kernel runs to completion with unspecified output.  SYNCHRONISES the device.
+ * Returns TRDQ_OK (word was 0), TRDQ_ERR_TIMEOUT, or TRDQ_ERR_CUDA; `*word` (may be NULL)
+ * receives the raw bits. */
+trdq_status trdq_device_status(uint32_t* word);
+
+/* Library version, major * 100 + minor. */
+int32_t trdq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRDQ_H_ */

@@ -1,0 +1,313 @@
+// Host side of the C ABI: argument validation, the time-step -> group table, object
+// lifetime, tensor-map encoding and the device status word.  No arithmetic of the method
+// happens here except the fused per-channel vectors, which are formed once per group.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace trdq {
+
+// One status word per device, written by kernels whose bounded waits expire.
+__device__ uint32_t g_status_word;
+
+uint32_t* device_status_word() {
+  static uint32_t* cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<uint32_t*>(p);
+  }
+  return cached[dev];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+trdq_status encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
+                                 uint64_t row_stride_bytes, uint32_t box_bytes, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return TRDQ_ERR_CUDA;
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_stride_bytes};
+  const cuuint32_t box[2] = {box_bytes, box_rows};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int find_group(const std::vector<int32_t>& bounds, int32_t t) {
+  const int G = static_cast<int>(bounds.size()) - 1;
+  for (int g = 0; g < G; ++g)
+    if (bounds[g] <= t && t < bounds[g + 1]) return g;
+  return -1;
+}
+
+}  // namespace trdq
+
+using namespace trdq;
+
+extern "C" {
+
+const char* trdq_status_string(trdq_status s) {
+  switch (s) {
+    case TRDQ_OK: return "ok";
+    case TRDQ_ERR_NULL: return "null pointer";
+    case TRDQ_ERR_SHAPE: return "unsupported shape";
+    case TRDQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case TRDQ_ERR_TIMESTEP: return "time-step outside the covered range";
+    case TRDQ_ERR_GROUP: return "invalid group specification";
+    case TRDQ_ERR_WBITS: return "unsupported weight bit-width";
+    case TRDQ_ERR_CUDA: return "CUDA call failed";
+    case TRDQ_ERR_NOMEM: return "out of memory";
+    case TRDQ_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case TRDQ_ERR_MISMATCH: return "objects do not belong together";
+  }
+  return "unknown status";
+}
+
+int32_t trdq_version(void) { return 100; }
+
+trdq_status trdq_rotation_create(const trdq_rotation_spec* spec, trdq_rotation** out) {
+  if (!spec || !out || !spec->t_bounds || !spec->signs) return TRDQ_ERR_NULL;
+  if (spec->block != TRDQ_BLOCK || spec->K <= 0 || spec->K % TRDQ_BLOCK != 0 || spec->K > TRDQ_MAX_K) return TRDQ_ERR_SHAPE;
+  if (spec->num_groups < 1) return TRDQ_ERR_GROUP;
+  const int G = spec->num_groups, K = spec->K;
+  for (int g = 0; g < G; ++g)
+    if (spec->t_bounds[g] >= spec->t_bounds[g + 1]) return TRDQ_ERR_GROUP;
+  const size_t n = static_cast<size_t>(G) * K;
+  for (size_t i = 0; i < n; ++i) {
+    if (spec->signs[i] != 1 && spec->signs[i] != -1) return TRDQ_ERR_GROUP;
+    if (spec->smooth && !(spec->smooth[i] > 0.0f && std::isfinite(spec->smooth[i]))) return TRDQ_ERR_GROUP;
+  }
+
+  trdq_rotation* rot = new (std::nothrow) trdq_rotation;
+  if (!rot) return TRDQ_ERR_NOMEM;
+  rot->K = K;
+  rot->num_groups = G;
+  rot->t_bounds.assign(spec->t_bounds, spec->t_bounds + G + 1);
+
+  // d * Delta / sqrt(128) and d / (Delta * sqrt(128)), in double, rounded once to fp32
+  const double norm = 0x1.6a09e667f3bcdp-4;  // 2^-3.5 = sqrt(2)/16, correctly rounded
+  std::vector<float> act(n), wv(n);
+  for (size_t i = 0; i < n; ++i) {
+    const double d = static_cast<double>(spec->signs[i]);
+    const double delta = spec->smooth ? static_cast<double>(spec->smooth[i]) : 1.0;
+    act[i] = static_cast<float>(d * delta * norm);
+    wv[i] = static_cast<float>(d / delta * norm);
+  }
+  if (cudaGetDevice(&rot->device) != cudaSuccess) {
+    delete rot;
+    return TRDQ_ERR_CUDA;
+  }
+  if (cudaMalloc(&rot->act_vec, n * sizeof(float)) != cudaSuccess || cudaMalloc(&rot->weight_vec, n * sizeof(float)) != cudaSuccess) {
+    cudaGetLastError();
+    trdq_rotation_destroy(rot);
+    return TRDQ_ERR_NOMEM;
+  }
+  if (cudaMemcpy(rot->act_vec, act.data(), n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(rot->weight_vec, wv.data(), n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+    trdq_rotation_destroy(rot);
+    return TRDQ_ERR_CUDA;
+  }
+  *out = rot;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_rotation_destroy(trdq_rotation* rot) {
+  if (!rot) return TRDQ_OK;
+  if (rot->act_vec) cudaFree(rot->act_vec);
+  if (rot->weight_vec) cudaFree(rot->weight_vec);
+  delete rot;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_find_group(const int32_t* t_bounds, int32_t num_groups, int32_t t, int32_t* g) {
+  if (!t_bounds || !g) return TRDQ_ERR_NULL;
+  if (num_groups < 1) return TRDQ_ERR_GROUP;
+  for (int i = 0; i < num_groups; ++i)
+    if (t_bounds[i] >= t_bounds[i + 1]) return TRDQ_ERR_GROUP;
+  for (int i = 0; i < num_groups; ++i)
+    if (t_bounds[i] <= t && t < t_bounds[i + 1]) {
+      *g = i;
+      return TRDQ_OK;
+    }
+  return TRDQ_ERR_TIMESTEP;
+}
+
+trdq_status trdq_group_of(const trdq_rotation* rot, int32_t t, int32_t* g) {
+  if (!rot || !g) return TRDQ_ERR_NULL;
+  const int r = find_group(rot->t_bounds, t);
+  if (r < 0) return TRDQ_ERR_TIMESTEP;
+  *g = r;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, int32_t N, int32_t wbits, trdq_weights** out,
+                                 void* stream) {
+  if (!rot || !W_bf16 || !out) return TRDQ_ERR_NULL;
+  if (wbits != 8 && wbits != 4) return TRDQ_ERR_WBITS;
+  if (N <= 0 || N % 16 != 0) return TRDQ_ERR_SHAPE;
+  if (!aligned16(W_bf16)) return TRDQ_ERR_ALIGN;
+  const int K = rot->K, G = rot->num_groups;
+
+  trdq_weights* w = new (std::nothrow) trdq_weights;
+  if (!w) return TRDQ_ERR_NOMEM;
+  w->N = N;
+  w->K = K;
+  w->wbits = wbits;
+  w->num_groups = G;
+  w->t_bounds = rot->t_bounds;
+  w->groups.resize(G);
+  if (cudaGetDevice(&w->device) != cudaSuccess) {
+    delete w;
+    return TRDQ_ERR_CUDA;
+  }
+  const size_t code_bytes = wbits == 8 ? static_cast<size_t>(N) * K : static_cast<size_t>(N) * K / 2;
+  const size_t scale_count = wbits == 8 ? static_cast<size_t>(N) : static_cast<size_t>(N) * (K / TRDQ_BLOCK);
+  const uint64_t row_bytes = wbits == 8 ? K : K / 2;
+  const uint32_t box_bytes = wbits == 8 ? 128 : 64;
+  for (int g = 0; g < G; ++g) {
+    GroupWeights& gw = w->groups[g];
+    if (cudaMalloc(&gw.codes, code_bytes) != cudaSuccess || cudaMalloc(&gw.scales, scale_count * sizeof(float)) != cudaSuccess) {
+      cudaGetLastError();
+      trdq_weights_destroy(w);
+      return TRDQ_ERR_NOMEM;
+    }
+    const cudaError_t e = launch_rotate_quantize(W_bf16, K, N, K, rot->weight_vec + static_cast<size_t>(g) * K, wbits == 8 ? 0 : 1,
+                                                 gw.codes, gw.scales, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+      trdq_weights_destroy(w);
+      return TRDQ_ERR_CUDA;
+    }
+    for (int i = 0; i < kNumTileN; ++i) {
+      const uint32_t box_rows = wbits == 8 ? kTileN[i] : 128;
+      const trdq_status st = encode_tmap_u8_sw128(&gw.tmap_b[i], gw.codes, row_bytes, N, row_bytes, box_bytes, box_rows);
+      if (st != TRDQ_OK) {
+        trdq_weights_destroy(w);
+        return st;
+      }
+    }
+  }
+  *out = w;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_weights_destroy(trdq_weights* w) {
+  if (!w) return TRDQ_OK;
+  for (auto& gw : w->groups) {
+    if (gw.codes) cudaFree(gw.codes);
+    if (gw.scales) cudaFree(gw.scales);
+  }
+  delete w;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_weights_info(const trdq_weights* w, int32_t* N, int32_t* K, int32_t* wbits, int32_t* num_groups) {
+  if (!w) return TRDQ_ERR_NULL;
+  if (N) *N = w->N;
+  if (K) *K = w->K;
+  if (wbits) *wbits = w->wbits;
+  if (num_groups) *num_groups = w->num_groups;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_weights_view(const trdq_weights* w, int32_t g, const void** Wq, const float** scales) {
+  if (!w) return TRDQ_ERR_NULL;
+  if (g < 0 || g >= w->num_groups) return TRDQ_ERR_GROUP;
+  if (Wq) *Wq = w->groups[g].codes;
+  if (scales) *scales = w->groups[g].scales;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, int8_t* codes,
+                                 float* scales, void* stream) {
+  if (!rot) return TRDQ_ERR_NULL;
+  if (M < 0) return TRDQ_ERR_SHAPE;
+  const int g = find_group(rot->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (M == 0) return TRDQ_OK;
+  if (!X_bf16 || !codes || !scales) return TRDQ_ERR_NULL;
+  if (ldx < rot->K) return TRDQ_ERR_SHAPE;
+  if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return TRDQ_ERR_ALIGN;
+  const cudaError_t e = launch_rotate_quantize(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, 0, codes,
+                                               scales, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
+                                 const int32_t M[2], const void* bias, void* const Y[2], const int64_t ld[2], bool raw,
+                                 void* stream) {
+  if (!w || !codes || !M || !Y || !ld || (!raw && !scales)) return TRDQ_ERR_NULL;
+  if (M[0] < 0 || M[1] < 0) return TRDQ_ERR_SHAPE;
+  const int g = find_group(w->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (raw && w->wbits != 8) return TRDQ_ERR_WBITS;
+  GemmSegment seg[2];
+  const int ld_mult = raw ? 4 : 8;
+  for (int s = 0; s < 2; ++s) {
+    seg[s] = GemmSegment{codes[s], raw ? nullptr : scales[s], Y[s], ld[s], M[s]};
+    if (M[s] == 0) continue;
+    if (!codes[s] || !Y[s] || (!raw && !scales[s])) return TRDQ_ERR_NULL;
+    if (ld[s] < w->N) return TRDQ_ERR_SHAPE;
+    if (ld[s] % ld_mult != 0 || !aligned16(codes[s]) || !aligned16(Y[s])) return TRDQ_ERR_ALIGN;
+  }
+  if (M[0] == 0 && M[1] == 0) return TRDQ_OK;
+  if (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)) return TRDQ_ERR_ALIGN;
+  if (w->wbits == 8) return launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream));
+  return launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream));
+}
+
+trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M, const void* bias_bf16,
+                        void* Y_bf16, int64_t ldy, void* stream) {
+  const int8_t* c[2] = {codes, nullptr};
+  const float* s[2] = {scales, nullptr};
+  const int32_t m[2] = {M, 0};
+  void* y[2] = {Y_bf16, nullptr};
+  const int64_t l[2] = {ldy, ldy};
+  return linear_common(w, t, c, s, m, bias_bf16, y, l, false, stream);
+}
+
+trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
+                            const int32_t M[2], const void* bias_bf16, void* const Y_bf16[2], const int64_t ldy[2], void* stream) {
+  return linear_common(w, t, codes, scales, M, bias_bf16, Y_bf16, ldy, false, stream);
+}
+
+trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes, int32_t M, int32_t* acc, int64_t ldacc, void* stream) {
+  const int8_t* c[2] = {codes, nullptr};
+  const int32_t m[2] = {M, 0};
+  void* y[2] = {acc, nullptr};
+  const int64_t l[2] = {ldacc, ldacc};
+  return linear_common(w, t, c, nullptr, m, nullptr, y, l, true, stream);
+}
+
+trdq_status trdq_device_status(uint32_t* word) {
+  uint32_t v = 0, zero = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return TRDQ_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof v) != cudaSuccess) return TRDQ_ERR_CUDA;
+  if (v != 0 && cudaMemcpyToSymbol(g_status_word, &zero, sizeof zero) != cudaSuccess) return TRDQ_ERR_CUDA;
+  if (word) *word = v;
+  return v == 0 ? TRDQ_OK : TRDQ_ERR_TIMEOUT;
+}
+
+}  // extern "C"

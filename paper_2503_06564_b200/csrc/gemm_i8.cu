@@ -1,0 +1,354 @@
+// INT8 x INT8 -> INT32 GEMM of Eq. 10 (G_t(X) . H_t(W) on the integer codes) with the
+// dequantizing epilogue  y = acc * sx[m] * sw[n] + bias[n]  ->  bf16.
+//
+// Persistent, warp-specialised kernel for sm_100a, one CTA per SM:
+//   warp 0      TMA producer: 128 x 128-byte tiles of the activation codes (A) and BN x 128-byte
+//               tiles of the weight codes (B), 128-byte swizzle, into a ring of shared-memory stages
+//   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction,
+//               four per stage); accumulators live in tensor memory, two stages of BN columns
+//   warp 2      allocates / frees tensor memory
+//   warps 4-7   epilogue: tcgen05.ld of the finished accumulator (warp q reads lanes 32q..32q+31,
+//               one output row per thread), fp32 dequantization, bf16 pack, 16-byte stores
+// The epilogue of tile i overlaps the main loop of tile i+1 through the second accumulator.
+// Tiles are visited column-block major so that concurrently running CTAs share one weight
+// tile; both CFG row segments are part of the same tile list, so a weight tile is fetched
+// once for both.  Every wait is bounded (see BoundedWaiter).
+#include <cuda_bf16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace trdq {
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kTileKBytes = 128;  // one swizzle atom: 128 int8 along K per stage
+constexpr int kUmmaK = 32;        // K of one kind::i8 instruction
+constexpr int kThreads = 256;
+constexpr int kEpilogueThreads = 128;
+constexpr int kAccStride = 256;   // tensor-memory columns between the two accumulator stages
+constexpr int kTmemCols = 512;
+constexpr int kSmemBudget = 227 * 1024;
+
+template <int BN>
+struct Cfg {
+  static constexpr int kABytes = kTileM * kTileKBytes;
+  static constexpr int kBBytes = BN * kTileKBytes;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  // parameters staged for the epilogue: (sw, bias) per column, one buffer per accumulator stage
+  static constexpr int kParamBytes = 2 * BN * 8;
+  static constexpr int kBarrierBytes = 256;
+  static constexpr int kStages = (kSmemBudget - 1024 - kParamBytes - kBarrierBytes) / kStageBytes;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kParamBytes + kBarrierBytes;
+  static_assert(kStages >= 3, "pipeline too shallow");
+  static_assert(kStages <= 12, "barrier area too small");
+};
+
+struct alignas(64) GemmParams {
+  CUtensorMap tmap_a[2];
+  CUtensorMap tmap_b;
+  const float* sx[2];
+  void* out[2];
+  int64_t ld[2];
+  int32_t M[2];
+  int32_t tiles_m[2];
+  const float* sw;
+  const __nv_bfloat16* bias;
+  int32_t N, K, tiles_n;
+  uint32_t* status;
+};
+
+struct TileCoord {
+  int seg, m0, n0;
+};
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int bn) {
+  const int tiles_m = p.tiles_m[0] + p.tiles_m[1];
+  const int nt = tile / tiles_m;
+  int mt = tile - nt * tiles_m;
+  TileCoord c;
+  c.seg = mt >= p.tiles_m[0] ? 1 : 0;
+  if (c.seg) mt -= p.tiles_m[0];
+  c.m0 = mt * kTileM;
+  c.n0 = nt * bn;
+  return c;
+}
+
+// MODE 0: bf16 dequantizing epilogue.  MODE 1: raw int32 accumulators.
+template <int BN, int MODE>
+__global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_constant__ GemmParams p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  float2* param_buf = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes + C::kParamBytes);
+  // barrier layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then the tensor-memory base address
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8 * C::kStages;
+  const uint32_t bar_tfull = bar_empty + 8 * C::kStages;
+  const uint32_t bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::kStages + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_tiles = (p.tiles_m[0] + p.tiles_m[1]) * p.tiles_n;
+  const int num_kb = p.K / kTileKBytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, kEpilogueThreads / 32);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tensormap(&p.tmap_a[0]);
+      prefetch_tensormap(&p.tmap_a[1]);
+      prefetch_tensormap(&p.tmap_b);
+      BoundedWaiter w(p.status, kStatusTimeoutProducer);
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(p, tile, BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          w.wait(bar_empty + 8 * stage, phase ^ 1);
+          const uint32_t a_dst = smem_base + stage * C::kStageBytes;
+          const uint32_t b_dst = a_dst + C::kABytes;
+          mbar_arrive_expect_tx(bar_full + 8 * stage, C::kStageBytes);
+          tma_load_2d(a_dst, &p.tmap_a[tc.seg], kb * kTileKBytes, tc.m0, bar_full + 8 * stage);
+          tma_load_2d(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0, bar_full + 8 * stage);
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+      }
+      w.settle();
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (elect_one()) {
+      BoundedWaiter w(p.status, kStatusTimeoutMma);
+      constexpr uint32_t idesc = umma_idesc_s8(BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        w.wait(bar_tempty + 8 * acc, acc_phase ^ 1);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kAccStride;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          w.wait(bar_full + 8 * stage, phase);
+          tc_fence_after();
+          const uint32_t a_addr = smem_base + stage * C::kStageBytes;
+          const uint64_t a_desc = umma_desc_k_sw128(a_addr);
+          const uint64_t b_desc = umma_desc_k_sw128(a_addr + C::kABytes);
+#pragma unroll
+          for (int k = 0; k < kTileKBytes / kUmmaK; ++k) {
+            // +32 bytes along K inside the swizzle atom = +2 in the 16-byte address field
+            umma_i8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+        umma_commit(bar_tfull + 8 * acc);  // accumulator complete
+        if (++acc == 2) {
+          acc = 0;
+          acc_phase ^= 1;
+        }
+      }
+      w.settle();
+    }
+  } else if (warp >= 4) {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp - 4;                 // lane quarter of tensor memory this warp may read
+    const int et = threadIdx.x - 4 * 32;    // 0..127
+    BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const TileCoord tc = tile_coord(p, tile, BN);
+      float2* pb = param_buf + acc * BN;
+      if (MODE == 0) {
+        for (int c = et; c < BN; c += kEpilogueThreads) {
+          const int n = tc.n0 + c;
+          float2 v = make_float2(0.0f, 0.0f);
+          if (n < p.N) {
+            v.x = __ldg(p.sw + n);
+            v.y = p.bias ? __bfloat162float(p.bias[n]) : 0.0f;
+          }
+          pb[c] = v;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+      }
+      const int row = tc.m0 + q * 32 + lane;
+      const bool row_ok = row < p.M[tc.seg];
+      const float sxm = (MODE == 0 && row_ok) ? __ldg(p.sx[tc.seg] + row) : 0.0f;
+
+      w.wait(bar_tfull + 8 * acc, acc_phase);
+      __syncwarp();
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccStride;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(t_row + c * 32, r);
+        tmem_wait_ld();
+        const int n_base = tc.n0 + c * 32;
+        if (!row_ok) continue;
+        if (MODE == 0) {
+          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out[tc.seg]) + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float y[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const float2 sb = pb[c * 32 + j + e];
+              const int32_t a = static_cast<int32_t>(r[j + e]);
+              const float af = static_cast<float>(a);
+              // sx*sw as an unevaluated sum s_hi + s_lo (exact), so that a cancellation between
+              // the product and the bias does not expose the rounding of the scale product
+              const float s_hi = __fmul_rn(sxm, sb.x);
+              const float s_lo = __fmaf_rn(sxm, sb.x, -s_hi);
+              float v = __fmaf_rn(af, s_lo, __fmaf_rn(af, s_hi, sb.y));
+              if (fabsf(af) >= 16777216.0f) v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
+              y[e] = v;
+            }
+            const __nv_bfloat162 h = __floats2bfloat162_rn(y[0], y[1]);
+            packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (n_base + 8 * v < p.N)
+              *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+          }
+        } else {
+          int32_t* out = static_cast<int32_t*>(p.out[tc.seg]) + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            if (n_base + 4 * v < p.N)
+              *reinterpret_cast<uint4*>(out + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+      if (++acc == 2) {
+        acc = 0;
+        acc_phase ^= 1;
+      }
+    }
+    w.settle();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+template <int BN, int MODE>
+cudaError_t launch_one(const GemmParams& p, int grid, cudaStream_t stream) {
+  using C = Cfg<BN>;
+  static bool configured[16] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 16 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_w8a8_kernel<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  gemm_w8a8_kernel<BN, MODE><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
+  return cudaGetLastError();
+}
+
+// Cost model for the tile width: waves of CTAs times the time of one tile (main loop grows
+// with BN; the 128-row operand and the fixed per-tile overhead do not).
+int choose_tile_n(int64_t tiles_m, int N, int sms) {
+  int best = 0;
+  double best_cost = 1e300;
+  for (int i = 0; i < kNumTileN; ++i) {
+    const int bn = kTileN[i];
+    const int64_t tiles = tiles_m * ((N + bn - 1) / bn);
+    const int64_t waves = (tiles + sms - 1) / sms;
+    const double cost = static_cast<double>(waves) * (bn + 24.0);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = i;
+    }
+  }
+  return best;
+}
+
+}  // namespace
+
+trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
+                           cudaStream_t stream) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+
+  GemmParams p;
+  int64_t tiles_m = 0;
+  for (int s = 0; s < 2; ++s) {
+    p.sx[s] = seg[s].sx;
+    p.out[s] = seg[s].out;
+    p.ld[s] = seg[s].ld;
+    p.M[s] = seg[s].M;
+    p.tiles_m[s] = (seg[s].M + kTileM - 1) / kTileM;
+    tiles_m += p.tiles_m[s];
+  }
+  if (tiles_m == 0) return TRDQ_OK;
+  const int ti = choose_tile_n(tiles_m, w->N, sms);
+  const int bn = kTileN[ti];
+  for (int s = 0; s < 2; ++s) {
+    // an empty segment still needs a valid descriptor object; reuse the other segment's
+    const GemmSegment& src = seg[s].M > 0 ? seg[s] : seg[1 - s];
+    trdq_status st = encode_tmap_u8_sw128(&p.tmap_a[s], src.codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(src.M),
+                                          static_cast<uint64_t>(w->K), kTileKBytes, kTileM);
+    if (st != TRDQ_OK) return st;
+  }
+  p.tmap_b = w->groups[g].tmap_b[ti];
+  p.sw = w->groups[g].scales;
+  p.bias = static_cast<const __nv_bfloat16*>(bias_bf16);
+  p.N = w->N;
+  p.K = w->K;
+  p.tiles_n = (w->N + bn - 1) / bn;
+  p.status = device_status_word();
+  if (!p.status) return TRDQ_ERR_CUDA;
+  const int64_t total = tiles_m * p.tiles_n;
+  const int grid = static_cast<int>(total < sms ? total : sms);
+
+  cudaError_t e;
+  if (raw_i32) {
+    e = bn == 128 ? launch_one<128, 1>(p, grid, stream) : bn == 192 ? launch_one<192, 1>(p, grid, stream) : launch_one<256, 1>(p, grid, stream);
+  } else {
+    e = bn == 128 ? launch_one<128, 0>(p, grid, stream) : bn == 192 ? launch_one<192, 0>(p, grid, stream) : launch_one<256, 0>(p, grid, stream);
+  }
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+}  // namespace trdq

@@ -1,0 +1,68 @@
+// Internal declarations shared by the translation units of the library (not installed).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/trdq.h"
+
+struct trdq_rotation {
+  int32_t K = 0;
+  int32_t num_groups = 0;
+  int device = 0;
+  std::vector<int32_t> t_bounds;  // host [G+1]
+  float* act_vec = nullptr;       // dev [G][K]: d * Delta * 2^-3.5
+  float* weight_vec = nullptr;    // dev [G][K]: d / Delta * 2^-3.5
+};
+
+namespace trdq {
+
+// Candidate accumulator tile widths of the GEMM (columns of Y per CTA tile).
+constexpr int kNumTileN = 3;
+constexpr int kTileN[kNumTileN] = {128, 192, 256};
+
+struct GroupWeights {
+  void* codes = nullptr;                // dev int8 [N,K] or packed uint8 [N,K/2]
+  float* scales = nullptr;              // dev fp32 [N] or [N,K/128]
+  CUtensorMap tmap_b[kNumTileN];        // TMA descriptors of `codes`, one per tile width
+};
+
+}  // namespace trdq
+
+struct trdq_weights {
+  int32_t N = 0, K = 0, wbits = 8, num_groups = 0;
+  int device = 0;
+  std::vector<int32_t> t_bounds;
+  std::vector<trdq::GroupWeights> groups;
+};
+
+namespace trdq {
+
+uint32_t* device_status_word();  // device address of the status word of the current device (nullptr on failure)
+
+// rotate_quantize.cu
+// mode 0: per-row int8 codes + fp32 scale per row; mode 1: per-128-block int4 codes packed + scale per block
+cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
+                                   void* codes, float* scales, cudaStream_t stream);
+
+// gemm_i8.cu
+struct GemmSegment {
+  const int8_t* codes;  // dev [M,K]
+  const float* sx;      // dev [M]
+  void* out;            // dev bf16 [M,ld] (or int32 [M,ld] for the raw mode)
+  int64_t ld;
+  int32_t M;
+};
+trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
+                           cudaStream_t stream);
+trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
+                           cudaStream_t stream);
+
+// tensor maps (driver entry point fetched through the runtime; no link-time libcuda dependency)
+// 2-D uint8 row-major [rows, row_bytes-wide], box = 128 bytes x box_rows, 128-byte swizzle.
+trdq_status encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
+                                 uint64_t row_stride_bytes, uint32_t box_bytes, uint32_t box_rows);
+
+}  // namespace trdq

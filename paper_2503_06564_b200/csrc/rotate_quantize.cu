@@ -1,0 +1,231 @@
+// Fused online transform + dynamic quantizer (Sec. 3.2 Eq. 10, G_t; Sec. 3.1 Eq. 1-2):
+// scale by the group's fused vector, rotate every 128-block with a Walsh-Hadamard butterfly
+// held in registers, take the absmax of the row (or of the block for 4-bit weights), and
+// emit integer codes.  One read of the input, one write of the codes; the rotated values
+// never leave the register file.
+//
+// Work decomposition.  A group of 8 consecutive lanes owns one 128-block of one row: lane l
+// holds elements 16*l .. 16*l+15 (two 16-byte loads).  Butterfly stages h = 1, 2, 4, 8 pair
+// registers of one thread; stages h = 16, 32, 64 pair lanes l ^ 1, l ^ 2, l ^ 4 by warp
+// shuffle.  All additions are separately rounded fp32 operations in this fixed order.
+// A CTA owns `rows` consecutive rows at a time (rows * K/128 groups); the row absmax is
+// combined through a shared-memory atomic max on the (non-negative) float bit patterns.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace trdq {
+namespace {
+
+constexpr int kLanesPerBlock = 8;
+constexpr int kElemsPerLane = 16;
+
+__device__ __forceinline__ void load_scaled16(const uint4* src, const float (&vec)[16], float (&u)[16]) {
+  const uint4 a = __ldg(src);
+  const uint4 b = __ldg(src + 1);
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    // bf16 -> fp32 is exact: the 16 bits become the high half of the fp32 pattern
+    const float lo = __uint_as_float(w[i] << 16);
+    const float hi = __uint_as_float(w[i] & 0xFFFF0000u);
+    u[2 * i] = __fmul_rn(lo, vec[2 * i]);
+    u[2 * i + 1] = __fmul_rn(hi, vec[2 * i + 1]);
+  }
+}
+
+// 128-point unnormalised Walsh-Hadamard transform across the 8 lanes of a group, natural
+// (Sylvester) order: stage h maps (a, b) = (u[i], u[i+h]) to (a + b, a - b).
+__device__ __forceinline__ void wht128(float (&u)[16], int lane8) {
+#pragma unroll
+  for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if ((i & h) == 0) {
+        const float a = u[i];
+        const float b = u[i + h];
+        u[i] = __fadd_rn(a, b);
+        u[i + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+#pragma unroll
+  for (int mask = 1; mask < 8; mask <<= 1) {
+    const bool upper = (lane8 & mask) != 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float other = __shfl_xor_sync(0xffffffffu, u[i], mask);
+      // lower lane: a + b with a = own; upper lane: a - b with a = other, b = own
+      u[i] = __fadd_rn(other, upper ? -u[i] : u[i]);
+    }
+  }
+}
+
+__device__ __forceinline__ float absmax16(const float (&u)[16]) {
+  float m = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(u[i]));
+  return m;
+}
+
+__device__ __forceinline__ float group_max(float m) {
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+  return m;
+}
+
+// Symmetric quantizer of Eq. 1 with z = 0: q = rne(v * fl(qmax / amax)).
+__device__ __forceinline__ int quantize_one(float v, float inv) { return __float2int_rn(__fmul_rn(v, inv)); }
+
+// MODE 0: int8 per row.  MODE 1: int4 per 128-block, packed.
+// P = blocks handled by one lane group per tile (P > 1 only for very wide rows).
+template <int MODE, int P>
+__global__ void __launch_bounds__(1024) rotate_quantize_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K,
+                                                               const float* __restrict__ vec, int8_t* __restrict__ codes,
+                                                               uint8_t* __restrict__ packed, float* __restrict__ scales,
+                                                               int32_t rows_per_tile, int32_t groups) {
+  __shared__ unsigned int row_max[3][32];
+  const int nb = K / TRDQ_BLOCK;
+  const int lane8 = threadIdx.x & (kLanesPerBlock - 1);
+  const int group = threadIdx.x / kLanesPerBlock;
+  const int items = rows_per_tile * nb;
+
+  if (MODE == 0) {
+    if (threadIdx.x < 32) row_max[0][threadIdx.x] = 0u;
+    __syncthreads();
+  }
+
+  // per-item placement inside a tile (fixed over the tile loop)
+  int r_of[P], b_of[P];
+  bool active[P];
+  float vreg[P][16];
+#pragma unroll
+  for (int p = 0; p < P; ++p) {
+    const int item = group + p * groups;
+    active[p] = (group < groups) && (item < items);
+    r_of[p] = active[p] ? item / nb : 0;
+    b_of[p] = active[p] ? item % nb : 0;
+    const float4* vp = reinterpret_cast<const float4*>(vec + b_of[p] * TRDQ_BLOCK + lane8 * kElemsPerLane);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 f = __ldg(vp + j);
+      vreg[p][4 * j] = f.x;
+      vreg[p][4 * j + 1] = f.y;
+      vreg[p][4 * j + 2] = f.z;
+      vreg[p][4 * j + 3] = f.w;
+    }
+  }
+
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  int it = 0;
+  for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    const int buf = it % 3;
+    if (MODE == 0 && threadIdx.x < 32) row_max[(it + 1) % 3][threadIdx.x] = 0u;
+
+    float u[P][16];
+    float gmax[P];
+    bool valid[P];
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+      const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r_of[p];
+      valid[p] = active[p] && row < M;
+      if (valid[p]) {
+        const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + b_of[p] * TRDQ_BLOCK + lane8 * kElemsPerLane);
+        load_scaled16(src, vreg[p], u[p]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[p][i] = 0.0f;
+      }
+    }
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+      wht128(u[p], lane8);
+      gmax[p] = group_max(absmax16(u[p]));
+      if (MODE == 0 && valid[p] && lane8 == 0) atomicMax(&row_max[buf][r_of[p]], __float_as_uint(gmax[p]));
+    }
+    if (MODE == 0) __syncthreads();
+
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+      if (!valid[p]) continue;
+      const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r_of[p];
+      const int64_t elem = row * K + b_of[p] * TRDQ_BLOCK + lane8 * kElemsPerLane;
+      if (MODE == 0) {
+        const float amax = __uint_as_float(row_max[buf][r_of[p]]);
+        const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+        uint32_t out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t word = 0;
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            int q = quantize_one(u[p][4 * j + b], inv);
+            q = max(-127, min(127, q));
+            word |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * b);
+          }
+          out[j] = word;
+        }
+        *reinterpret_cast<uint4*>(codes + elem) = make_uint4(out[0], out[1], out[2], out[3]);
+        if (b_of[p] == 0 && lane8 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
+      } else {
+        const float amax = gmax[p];
+        const float inv = amax > 0.0f ? __fdiv_rn(7.0f, amax) : 0.0f;
+        uint32_t out[2] = {0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          int q = quantize_one(u[p][i], inv);
+          q = max(-7, min(7, q));
+          out[i / 8] |= (static_cast<uint32_t>(q) & 0xFu) << (4 * (i % 8));  // even k -> low nibble of its byte
+        }
+        *reinterpret_cast<uint2*>(packed + elem / 2) = make_uint2(out[0], out[1]);
+        if (lane8 == 0) scales[row * nb + b_of[p]] = __fdiv_rn(amax, 7.0f);
+      }
+    }
+  }
+}
+
+template <int MODE, int P>
+cudaError_t launch(const void* x, int64_t ldx, int32_t M, int32_t K, const float* vec, void* codes, float* scales,
+                   int rows_per_tile, int groups, cudaStream_t stream) {
+  int threads = groups * kLanesPerBlock;
+  threads = (threads + 31) / 32 * 32;
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int ctas_per_sm = max(1, 2048 / threads);
+  const int grid = min(num_tiles, sms * ctas_per_sm);
+  rotate_quantize_kernel<MODE, P><<<grid, threads, 0, stream>>>(
+      static_cast<const __nv_bfloat16*>(x), ldx, M, K, vec, static_cast<int8_t*>(codes), static_cast<uint8_t*>(codes), scales,
+      rows_per_tile, groups);
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t dispatch(const void* x, int64_t ldx, int32_t M, int32_t K, const float* vec, void* codes, float* scales,
+                     cudaStream_t stream) {
+  const int nb = K / TRDQ_BLOCK;
+  if (nb <= 128) {
+    // about 32 lane groups (256 threads) per CTA, whole rows only, at most 32 rows per tile
+    int rows = 32 / nb;
+    if (rows < 1) rows = 1;
+    if (rows > 32) rows = 32;
+    return launch<MODE, 1>(x, ldx, M, K, vec, codes, scales, rows, rows * nb, stream);
+  }
+  const int p = (nb + 127) / 128;  // nb <= 1024 -> p <= 8
+  if (p <= 2) return launch<MODE, 2>(x, ldx, M, K, vec, codes, scales, 1, (nb + 1) / 2, stream);
+  if (p <= 4) return launch<MODE, 4>(x, ldx, M, K, vec, codes, scales, 1, (nb + 3) / 4, stream);
+  return launch<MODE, 8>(x, ldx, M, K, vec, codes, scales, 1, (nb + 7) / 8, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
+                                   void* codes, float* scales, cudaStream_t stream) {
+  if (M == 0) return cudaSuccess;
+  if (mode == 0) return dispatch<0>(x_bf16, ldx, M, K, vec, codes, scales, stream);
+  return dispatch<1>(x_bf16, ldx, M, K, vec, codes, scales, stream);
+}
+
+}  // namespace trdq

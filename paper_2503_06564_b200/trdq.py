@@ -1,0 +1,245 @@
+"""ctypes binding of ``libtrdq.so``: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (``include/trdq.h``)
+and does nothing but turn torch tensors into pointers, sizes and the current
+stream.  All arithmetic runs in the CUDA kernels of the library; if the shared
+object is missing the import of this module's library handle fails loudly, and
+there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtrdq.so")
+
+OK = 0
+STATUS_NAMES = {0: "TRDQ_OK", 1: "TRDQ_ERR_NULL", 2: "TRDQ_ERR_SHAPE", 3: "TRDQ_ERR_ALIGN", 4: "TRDQ_ERR_TIMESTEP",
+                5: "TRDQ_ERR_GROUP", 6: "TRDQ_ERR_WBITS", 7: "TRDQ_ERR_CUDA", 8: "TRDQ_ERR_NOMEM", 9: "TRDQ_ERR_TIMEOUT",
+                10: "TRDQ_ERR_MISMATCH"}
+
+EXPORTS = (
+    "trdq_status_string", "trdq_version", "trdq_rotation_create", "trdq_rotation_destroy", "trdq_group_of",
+    "trdq_find_group", "trdq_prepare_weights", "trdq_weights_destroy", "trdq_weights_info", "trdq_weights_view",
+    "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
+)
+
+
+class TrdqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {STATUS_NAMES.get(self.status, self.status)} ({status_string(self.status)})")
+
+
+class RotationSpec(C.Structure):
+    _fields_ = [("K", C.c_int32), ("block", C.c_int32), ("num_groups", C.c_int32),
+                ("t_bounds", C.POINTER(C.c_int32)), ("signs", C.POINTER(C.c_int8)), ("smooth", C.POINTER(C.c_float))]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Raises if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_06564_b200.build`")
+        l = C.CDLL(LIB_PATH)
+        l.trdq_status_string.restype = C.c_char_p
+        l.trdq_status_string.argtypes = [C.c_int]
+        l.trdq_version.restype = C.c_int32
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        l.trdq_rotation_create.argtypes = [C.POINTER(RotationSpec), C.POINTER(vp)]
+        l.trdq_rotation_destroy.argtypes = [vp]
+        l.trdq_group_of.argtypes = [vp, i32, C.POINTER(i32)]
+        l.trdq_find_group.argtypes = [C.POINTER(i32), i32, i32, C.POINTER(i32)]
+        l.trdq_prepare_weights.argtypes = [vp, vp, i32, i32, C.POINTER(vp), vp]
+        l.trdq_weights_destroy.argtypes = [vp]
+        l.trdq_weights_info.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        l.trdq_weights_view.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp)]
+        l.trdq_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp]
+        l.trdq_linear.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
+        l.trdq_linear_cfg.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), vp, C.POINTER(vp),
+                                      C.POINTER(i64), vp]
+        l.trdq_gemm_i32.argtypes = [vp, i32, vp, i32, vp, i64, vp]
+        l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().trdq_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise TrdqError(status, where)
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def trdq_find_group(t_bounds: Sequence[int], t: int) -> int:
+    b = np.ascontiguousarray(t_bounds, dtype=np.int32)
+    g = C.c_int32(-1)
+    _check(lib().trdq_find_group(b.ctypes.data_as(C.POINTER(C.c_int32)), len(b) - 1, int(t), C.byref(g)), "trdq_find_group")
+    return g.value
+
+
+class Rotation:
+    """Handle of a trdq_rotation (per-group device tables of one C_in)."""
+
+    def __init__(self, K: int, t_bounds, signs, smooth=None, block: int = 128):
+        self._h = C.c_void_p()
+        b = np.ascontiguousarray(t_bounds, dtype=np.int32)
+        s = np.ascontiguousarray(signs, dtype=np.int8)
+        sm = None if smooth is None else np.ascontiguousarray(smooth, dtype=np.float32)
+        spec = RotationSpec(int(K), int(block), int(len(b) - 1), b.ctypes.data_as(C.POINTER(C.c_int32)),
+                            s.ctypes.data_as(C.POINTER(C.c_int8)),
+                            None if sm is None else sm.ctypes.data_as(C.POINTER(C.c_float)))
+        _check(lib().trdq_rotation_create(C.byref(spec), C.byref(self._h)), "trdq_rotation_create")
+        self.K = int(K)
+        self.num_groups = int(len(b) - 1)
+
+    def group_of(self, t: int) -> int:
+        g = C.c_int32(-1)
+        _check(lib().trdq_group_of(self._h, int(t), C.byref(g)), "trdq_group_of")
+        return g.value
+
+    def close(self) -> None:
+        if self._h:
+            lib().trdq_rotation_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Weights:
+    """Handle of a trdq_weights (H_t(W) of one layer, quantized for every group)."""
+
+    def __init__(self, handle: C.c_void_p):
+        self._h = handle
+        n, k, wb, g = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+        _check(lib().trdq_weights_info(self._h, C.byref(n), C.byref(k), C.byref(wb), C.byref(g)), "trdq_weights_info")
+        self.N, self.K, self.wbits, self.num_groups = n.value, k.value, wb.value, g.value
+
+    def view(self, g: int) -> Tuple[int, int]:
+        """(device pointer of the codes, device pointer of the scales) of group g."""
+        wq, sc = C.c_void_p(), C.c_void_p()
+        _check(lib().trdq_weights_view(self._h, int(g), C.byref(wq), C.byref(sc)), "trdq_weights_view")
+        return wq.value, sc.value
+
+    def view_tensors(self, g: int):
+        """Copies of group g's codes and scales as torch tensors (device)."""
+        import torch
+        wq, sc = self.view(g)
+        if self.wbits == 8:
+            codes = torch.empty((self.N, self.K), dtype=torch.int8, device="cuda")
+            scales = torch.empty((self.N,), dtype=torch.float32, device="cuda")
+        else:
+            codes = torch.empty((self.N, self.K // 2), dtype=torch.uint8, device="cuda")
+            scales = torch.empty((self.N, self.K // 128), dtype=torch.float32, device="cuda")
+        cudart = torch.cuda.cudart()
+        torch.cuda.current_stream().synchronize()
+        for dst, src in ((codes, wq), (scales, sc)):
+            err = cudart.cudaMemcpy(dst.data_ptr(), src, dst.numel() * dst.element_size(), 3)  # device -> device
+            if int(err) != 0:
+                raise RuntimeError(f"cudaMemcpy failed: {err}")
+        return codes, scales
+
+    def close(self) -> None:
+        if self._h:
+            lib().trdq_weights_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def trdq_prepare_weights(rot: Rotation, W_bf16, wbits: int = 8) -> Weights:
+    assert W_bf16.is_cuda and W_bf16.is_contiguous() and W_bf16.dim() == 2 and W_bf16.element_size() == 2
+    if W_bf16.shape[1] != rot.K:
+        raise TrdqError(2, "trdq_prepare_weights (K of W differs from the rotation's)")
+    h = C.c_void_p()
+    _check(lib().trdq_prepare_weights(rot._h, _ptr(W_bf16), int(W_bf16.shape[0]), int(wbits), C.byref(h), _stream()),
+           "trdq_prepare_weights")
+    return Weights(h)
+
+
+def trdq_rotate_quantize(rot: Rotation, t: int, X_bf16, codes=None, scales=None):
+    """codes int8 [M,K], scales fp32 [M] of the rotated activations at time-step t."""
+    import torch
+    assert X_bf16.is_cuda and X_bf16.dim() == 2 and X_bf16.element_size() == 2 and X_bf16.stride(1) == 1
+    M = int(X_bf16.shape[0])
+    if codes is None:
+        codes = torch.empty((M, rot.K), dtype=torch.int8, device=X_bf16.device)
+    if scales is None:
+        scales = torch.empty((M,), dtype=torch.float32, device=X_bf16.device)
+    ldx = int(X_bf16.stride(0)) if M > 1 else rot.K
+    _check(lib().trdq_rotate_quantize(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(codes), _ptr(scales), _stream()),
+           "trdq_rotate_quantize")
+    return codes, scales
+
+
+def trdq_linear(w: Weights, t: int, codes, scales, bias_bf16=None, out=None):
+    """bf16 [M,N] output of the integer GEMM with the dequantizing epilogue."""
+    import torch
+    M = int(codes.shape[0])
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.bfloat16, device=codes.device)
+    ldy = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_linear(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, _stream()),
+           "trdq_linear")
+    return out
+
+
+def trdq_linear_cfg(w: Weights, t: int, codes2, scales2, bias_bf16=None, out2=None):
+    """Two row segments (conditional, unconditional) through one launch."""
+    import torch
+    Ms = [int(c.shape[0]) for c in codes2]
+    if out2 is None:
+        out2 = [torch.empty((m, w.N), dtype=torch.bfloat16, device=codes2[0].device) for m in Ms]
+    vp2, i32_2, i64_2 = C.c_void_p * 2, C.c_int32 * 2, C.c_int64 * 2
+    _check(lib().trdq_linear_cfg(w._h, int(t), vp2(*[_ptr(c) for c in codes2]), vp2(*[_ptr(s) for s in scales2]),
+                                 i32_2(*Ms), _ptr(bias_bf16), vp2(*[_ptr(o) for o in out2]),
+                                 i64_2(*[int(o.stride(0)) if m > 1 else w.N for o, m in zip(out2, Ms)]), _stream()),
+           "trdq_linear_cfg")
+    return out2
+
+
+def trdq_gemm_i32(w: Weights, t: int, codes, out=None):
+    """Raw int32 accumulators [M,N] of the integer GEMM (8-bit weights only)."""
+    import torch
+    M = int(codes.shape[0])
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.int32, device=codes.device)
+    ld = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_gemm_i32(w._h, int(t), _ptr(codes), M, _ptr(out), ld, _stream()), "trdq_gemm_i32")
+    return out
+
+
+def trdq_device_status() -> int:
+    """Synchronises; returns the raw status word (0 = no bounded wait expired) and clears it."""
+    word = C.c_uint32(0)
+    st = lib().trdq_device_status(C.byref(word))
+    if st not in (0, 9):
+        raise TrdqError(st, "trdq_device_status")
+    return word.value

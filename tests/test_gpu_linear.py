@@ -1,0 +1,182 @@
+"""GPU parity: INT8 tcgen05 GEMM (raw accumulators and dequantizing epilogue) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from oracle import trdq_oracle as O
+from paper_2503_06564_b200 import workloads as WL
+from tests.util import bf16_to_f32_np, check_output, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(N, K, G, seed, wbits=8):
+    """A prepared layer on the device plus the oracle's own codes for every group."""
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(seed)
+    signs = (rng.integers(0, 2, (G, K)) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.5, 2.0, (G, K)).astype(np.float32)
+    bounds = WL.group_bounds(G)
+    rot = trdq.Rotation(K, bounds, signs, smooth)
+    w = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.02)
+    bias = WL.to_bf16_bits(rng.standard_normal(N) * 0.01)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(w), wbits)
+    ref = []
+    for g in range(G):
+        act, wv = O.fused_vectors(signs[g], smooth[g])
+        ref.append((act, *(O.prepare_w8(w, wv) if wbits == 8 else O.prepare_w4(w, wv))))
+    return rot, wts, bounds, bias, ref
+
+
+def _acts(M, K, seed):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((M, K))
+    x[:, rng.choice(K, max(1, K // 100), replace=False)] *= 30.0
+    return WL.to_bf16_bits(x)
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (256, 1024, 1024),     # single-layer configuration: two row tiles
+    (300, 1152, 1152),     # ragged rows, 9 k-blocks
+    (129, 3456, 1152),     # one row past a tile
+    (200, 1152, 4608),     # 36 k-blocks: the stage ring wraps many times
+    (1, 16, 128),          # smallest legal problem
+    (77, 1040, 256),       # N is not a multiple of any tile width
+    (520, 4608, 1152),
+])
+def test_int32_accumulators_bit_exact(M, N, K):
+    import torch
+    from paper_2503_06564_b200 import trdq
+    G = 2
+    rot, wts, bounds, _, ref = _setup(N, K, G, 100 + N + K)
+    x = _acts(M, K, 7 + M)
+    for g in range(G):
+        act, qw_ref, sw_ref = ref[g]
+        q_ref, _ = O.rotate_quantize(x, act)
+        # the GEMM is judged on the oracle's codes, so that only the contraction is under test
+        wq_dev, _ = wts.view_tensors(g)
+        assert np.array_equal(wq_dev.cpu().numpy(), qw_ref)
+        acc = trdq.trdq_gemm_i32(wts, int(bounds[g]), torch.from_numpy(q_ref).cuda())
+        acc_ref = O.gemm_i32(q_ref, qw_ref)
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    assert trdq.trdq_device_status() == 0
+
+
+def test_int32_accumulators_extreme_codes():
+    """All codes at +-127 with K = 4608: |acc| reaches 74 million (> 2^24), exact in int32."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    N, K, M = 64, 4608, 130
+    signs = np.ones((1, K), np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs, np.full((1, K), np.float32(2.0 ** 3.5), np.float32))
+    # weights whose rotated rows are +-c in every position: a single non-zero per 128-block
+    w = np.zeros((N, K))
+    rng = np.random.default_rng(0)
+    for n in range(N):
+        for b in range(K // 128):
+            w[n, b * 128 + rng.integers(0, 128)] = rng.choice([-1.0, 1.0])
+    wb = WL.to_bf16_bits(w)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(wb), 8)
+    _, wv = O.fused_vectors(signs[0], np.full(K, np.float32(2.0 ** 3.5), np.float32))
+    qw_ref, sw_ref = O.prepare_w8(wb, wv)
+    assert set(np.unique(qw_ref).tolist()) == {-127, 127}
+    q = (rng.integers(0, 2, (M, K)) * 254 - 127).astype(np.int8)
+    q[0] = qw_ref[0]                      # one row fully aligned with a weight row: acc = K * 127^2
+    acc = trdq.trdq_gemm_i32(wts, 0, torch.from_numpy(q).cuda()).cpu().numpy()
+    acc_ref = q.astype(np.int64) @ qw_ref.astype(np.int64).T
+    assert acc_ref[0, 0] == K * 127 * 127 and acc_ref.max() < 2 ** 31
+    assert np.array_equal(acc.astype(np.int64), acc_ref)
+    # epilogue on accumulators that do not fit fp32 exactly
+    sx = rng.uniform(0.01, 0.02, M).astype(np.float32)
+    y = trdq.trdq_linear(wts, 0, torch.from_numpy(q).cuda(), torch.from_numpy(sx).cuda())
+    y_ref = O.epilogue(acc_ref.astype(np.int32), sx, sw_ref, None)
+    check_output(bf16_to_f32_np(y), y_ref, max_ulp=1.0)
+
+
+@pytest.mark.parametrize("M,N,K,with_bias", [
+    (256, 1024, 1024, True),
+    (300, 1152, 1152, True),
+    (129, 3456, 1152, False),
+    (200, 1152, 4608, True),
+    (1, 16, 128, True),
+    (77, 1040, 256, True),
+])
+def test_linear_matches_oracle(M, N, K, with_bias):
+    import torch
+    from paper_2503_06564_b200 import trdq
+    G = 2
+    rot, wts, bounds, bias, ref = _setup(N, K, G, 200 + N + K)
+    x = _acts(M, K, 17 + M)
+    xd = to_dev_bf16(x)
+    bias_d = to_dev_bf16(bias) if with_bias else None
+    for g in range(G):
+        t = int(bounds[g])
+        act, qw_ref, sw_ref = ref[g]
+        q_ref, sx_ref = O.rotate_quantize(x, act)
+        codes, scales = trdq.trdq_rotate_quantize(rot, t, xd)
+        assert np.array_equal(codes.cpu().numpy(), q_ref) and np.array_equal(scales.cpu().numpy(), sx_ref)
+        y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
+        y_ref = O.linear_w8_rows(q_ref, sx_ref, qw_ref, sw_ref, bias if with_bias else None, np.arange(M))
+        l2, ulps = check_output(bf16_to_f32_np(y), y_ref, max_ulp=2.0, rel_l2=2e-3)
+        assert ulps <= 1.0      # the epilogue is accurate to half a bf16 step plus fp32 noise
+    assert trdq.trdq_device_status() == 0
+
+
+def test_epilogue_cancellation_against_bias():
+    """Outputs where acc*sx*sw and the bias cancel to almost nothing must still be within 2 bf16
+    steps of the exact value: the scale product is carried as an exact two-term sum."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    N, K, M = 16, 128, 128
+    signs = np.ones((1, K), np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs, np.full((1, K), np.float32(2.0 ** 3.5), np.float32))
+    w = np.zeros((N, K))
+    w[:, 0] = 1.0                                    # rotated rows are all ones -> codes all 127
+    wb = WL.to_bf16_bits(w)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(wb), 8)
+    _, wv = O.fused_vectors(signs[0], np.full(K, np.float32(2.0 ** 3.5), np.float32))
+    qw_ref, sw_ref = O.prepare_w8(wb, wv)
+    rng = np.random.default_rng(4)
+    q = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    acc = q.astype(np.int64) @ qw_ref.astype(np.int64).T
+    sx = rng.uniform(0.003, 0.03, M).astype(np.float32)
+    # bias = bf16 value closest to -acc*sx*sw of row n (so row n, column n nearly cancels)
+    exact = acc.astype(np.float64) * sx[:, None].astype(np.float64) * sw_ref[None, :].astype(np.float64)
+    bias = WL.to_bf16_bits(-np.diag(exact[:N, :N]))
+    y = trdq.trdq_linear(wts, 0, torch.from_numpy(q).cuda(), torch.from_numpy(sx).cuda(), to_dev_bf16(bias))
+    y_ref = O.epilogue(acc.astype(np.int32), sx, sw_ref, bias)
+    d = np.abs(np.diag(y_ref[:N, :N]))
+    assert (d < 1e-2 * np.abs(np.diag(exact[:N, :N]))).all()     # the cancellation really happens
+    check_output(bf16_to_f32_np(y), y_ref, max_ulp=2.0)
+
+
+def test_linear_strided_output_and_cfg_segments():
+    import torch
+    from paper_2503_06564_b200 import trdq
+    M, N, K = 300, 1152, 1152
+    rot, wts, bounds, bias, ref = _setup(N, K, 2, 321)
+    x = _acts(M, K, 3)
+    t = int(bounds[1])
+    codes, scales = trdq.trdq_rotate_quantize(rot, t, to_dev_bf16(x))
+    bias_d = to_dev_bf16(bias)
+    y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
+    # output rows with a larger stride; the padding must stay untouched
+    wide = torch.full((M, N + 24), 7.0, dtype=torch.bfloat16, device="cuda")
+    trdq.trdq_linear(wts, t, codes, scales, bias_d, out=wide[:, :N])
+    assert torch.equal(wide[:, :N], y) and bool((wide[:, N:] == 7.0).all())
+    # conditional / unconditional halves stored apart, one launch
+    mc = 171
+    halves = trdq.trdq_linear_cfg(wts, t, [codes[:mc].contiguous(), codes[mc:].contiguous()],
+                                  [scales[:mc].contiguous(), scales[mc:].contiguous()], bias_d)
+    assert torch.equal(torch.cat(halves), y)
+    empty = trdq.trdq_linear_cfg(wts, t, [codes[:0], codes], [scales[:0], scales], bias_d)
+    assert empty[0].shape[0] == 0 and torch.equal(empty[1], y)
+    # M == 0
+    assert trdq.trdq_linear(wts, t, codes[:0], scales[:0], bias_d).shape == (0, N)
+    # errors
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_linear(wts, 5000, codes, scales, bias_d)
+    assert e.value.status == 4
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_linear(wts, t, codes, scales, bias_d, out=torch.empty((M, N + 4), dtype=torch.bfloat16, device="cuda")[:, :N])
+    assert e.value.status == 3
+    assert trdq.trdq_device_status() == 0

@@ -1,0 +1,100 @@
+"""CPU-side checks of the C ABI: the shared library builds, loads without a GPU, exports every
+symbol the header declares, and validates arguments on the host before touching CUDA."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2503_06564_b200 import build, trdq
+    build.build()
+    return trdq.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2503_06564_b200 import trdq
+    header = open(os.path.join(ROOT, "include", "trdq.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(trdq_[a-z0-9_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(trdq.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    from paper_2503_06564_b200 import trdq
+    seen = set()
+    for code in range(0, 11):
+        s = trdq.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 11
+    assert trdq.status_string(99) == "unknown status"
+    assert lib.trdq_version() >= 100
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5])
+def test_find_group_exhaustive(lib, G):
+    from paper_2503_06564_b200 import trdq, workloads as WL
+    b = WL.group_bounds(G)
+    for t in range(1000):
+        g = trdq.trdq_find_group(b, t)
+        assert b[g] <= t < b[g + 1]
+    for t in (-1, 1000, 12345):
+        with pytest.raises(trdq.TrdqError) as e:
+            trdq.trdq_find_group(b, t)
+        assert e.value.status == 4
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_find_group([0, 10, 10], 5)
+    assert e.value.status == 5
+
+
+def test_host_side_validation_needs_no_device(lib):
+    """Bad specifications are rejected before any CUDA call, so the codes are the same on a CPU-only box."""
+    from paper_2503_06564_b200 import trdq
+    ones = np.ones((2, 256), np.int8)
+
+    def status_of(**kw):
+        args = dict(K=256, t_bounds=[0, 500, 1000], signs=ones, smooth=None, block=128)
+        args.update(kw)
+        try:
+            trdq.Rotation(**args)
+        except trdq.TrdqError as e:
+            return e.status
+        return 0
+
+    assert status_of(K=200) == 2
+    assert status_of(K=0) == 2
+    assert status_of(block=64) == 2
+    assert status_of(K=131072 + 128, signs=np.ones((2, 131072 + 128), np.int8)) == 2
+    assert status_of(t_bounds=[0, 500, 400]) == 5
+    bad = ones.copy()
+    bad[1, 5] = 0
+    assert status_of(signs=bad) == 5
+    assert status_of(smooth=np.zeros((2, 256), np.float32)) == 5
+    # null handles
+    g = C.c_int32()
+    assert lib.trdq_group_of(None, 0, C.byref(g)) == 1
+    assert lib.trdq_rotate_quantize(None, 0, None, 0, 0, None, None, None) == 1
+    assert lib.trdq_linear(None, 0, None, None, 0, None, None, 0, None) == 1
+    assert lib.trdq_weights_info(None, None, None, None, None) == 1
+    assert lib.trdq_rotation_destroy(None) == 0 and lib.trdq_weights_destroy(None) == 0
+    import torch
+    if not torch.cuda.is_available():
+        # a valid specification cannot be realised without a device, and says so
+        assert status_of() == 7
+
+
+def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):
+    from paper_2503_06564_b200 import trdq
+    monkeypatch.setattr(trdq, "_lib", None)
+    monkeypatch.setattr(trdq, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(ImportError):
+        trdq.lib()

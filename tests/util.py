@@ -1,0 +1,50 @@
+"""Helpers shared by the GPU parity tests: tensor transport and the comparison rules."""
+import numpy as np
+
+from paper_2503_06564_b200 import workloads as WL
+
+
+def to_dev_bf16(bits: np.ndarray):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def bf16_to_f32_np(t) -> np.ndarray:
+    """Device bf16 tensor -> host fp32 array (exact widening)."""
+    import torch
+    return WL.bf16_bits_to_f32(t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16))
+
+
+def bf16_ulp(y_ref: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 numbers (8 significant bits) at the magnitude of y_ref."""
+    _, e = np.frexp(np.abs(y_ref).astype(np.float64))
+    return np.ldexp(1.0, np.maximum(e - 8, -133))
+
+
+def check_codes(codes_gpu: np.ndarray, codes_ref: np.ndarray, v_ref: np.ndarray = None, inv_ref: np.ndarray = None):
+    """Integer codes: bit-exact, except that at most 1e-4 of them may differ by one step, and
+    only where the fp32 value before rounding lies within 1e-4 of a .5 boundary."""
+    diff = codes_gpu.astype(np.int32) - codes_ref.astype(np.int32)
+    bad = diff != 0
+    nbad = int(bad.sum())
+    if nbad == 0:
+        return 0
+    assert np.abs(diff).max() <= 1, f"codes differ by more than one step (max {np.abs(diff).max()})"
+    assert nbad <= 1e-4 * codes_ref.size, f"{nbad} of {codes_ref.size} codes differ"
+    if v_ref is not None and inv_ref is not None:
+        pre = (v_ref * inv_ref[:, None]).astype(np.float32)[bad]
+        frac = np.abs(pre - np.floor(pre) - 0.5)
+        assert frac.max() <= 1e-4, "a differing code is not at a rounding tie"
+    return nbad
+
+
+def check_output(y_gpu: np.ndarray, y_ref: np.ndarray, max_ulp: float = 2.0, rel_l2: float = 2e-3):
+    """bf16 outputs against the oracle's fp32 values: relative L2 error and max error in bf16 ulps."""
+    y_gpu = y_gpu.astype(np.float64)
+    y_ref64 = y_ref.astype(np.float64)
+    err = np.abs(y_gpu - y_ref64)
+    ulps = err / bf16_ulp(y_ref)
+    l2 = np.sqrt((err ** 2).sum()) / max(np.sqrt((y_ref64 ** 2).sum()), 1e-30)
+    assert l2 <= rel_l2, f"relative L2 error {l2:.3e} > {rel_l2}"
+    assert ulps.max() <= max_ulp, f"max error {ulps.max():.3f} bf16 ulp at {np.unravel_index(ulps.argmax(), ulps.shape)}"
+    return float(l2), float(ulps.max())
