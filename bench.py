@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the time-rotated quantized linear path on B200.
+
+A step is one denoising step of the DiT workload: for each of the transformer blocks, each of its
+quantized linears runs rotate + quantize and the INT8 GEMM with its epilogue (two kernels per
+linear), at the time-step of that sampling step, so the timed run includes the group switches.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2503_06564_b200 import workloads as WL
+
+METRIC = "rotated_w8a8_linear_tops"
+UNIT = "TOPS"
+INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def step_ops(wl: WL.Workload) -> float:
+    """Integer operations (2 per multiply-add) of one denoising step."""
+    total = 0.0
+    for layer in wl.layers:
+        total += 2.0 * wl.M * layer.N * layer.K
+    for layer in wl.extra_layers:
+        total += 2.0 * (layer.M or wl.M) * layer.N * layer.K
+    return total * wl.blocks
+
+
+def step_rq_bytes(wl: WL.Workload) -> float:
+    """Algorithmic bytes of the rotate + quantize launches of one step: 3K + 4 per token."""
+    total = 0.0
+    for layer in wl.layers + wl.extra_layers:
+        total += (layer.M or wl.M) * (3.0 * layer.K + 4.0)
+    return total * wl.blocks
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.device_index = device_index
+        self.proc = None
+        self.path = os.path.join(ROOT, "gpurun_out", f"clocks_rank{device_index}.csv")
+
+    def start(self):
+        try:
+            os.makedirs(os.path.dirname(self.path), exist_ok=True)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.device_index)], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# device workload
+# ------------------------------------------------------------------------------------------
+def make_device_x(wl: WL.Workload, M: int, K: int, gen):
+    """Activations drawn on the device with the recipe of workloads.make_x: N(0,1) bulk, 1 % of the
+    channels heavy tailed (Student-t, nu = 3) or scaled, per the workload."""
+    import torch
+    x = torch.randn((M, K), generator=gen, device="cuda", dtype=torch.float32)
+    n_out = int(np.ceil(0.01 * K))
+    ch = torch.randperm(K, generator=gen, device="cuda")[:n_out]
+    if wl.outlier == "student_t3":
+        z = torch.randn((M, n_out), generator=gen, device="cuda")
+        chi2 = (torch.randn((M, n_out, 3), generator=gen, device="cuda") ** 2).sum(-1)
+        x[:, ch] = z / torch.sqrt(chi2 / 3.0)
+    elif wl.outlier == "scale30":
+        x[:, ch] *= 30.0
+    elif wl.outlier == "fixed50":
+        x[:, ch] *= 50.0
+    return x.to(torch.bfloat16)
+
+
+def build_device_workload(wl: WL.Workload, seed: int, blocks: int):
+    """Distinct weights, activations and outputs for every linear of every block, so that one step
+    streams a working set far larger than L2."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    layers = trdq.LayerList()
+    alphas = WL.group_alphas(wl.num_groups)
+    rng = np.random.default_rng(seed)
+    for b in range(blocks):
+        for layer in wl.layers + wl.extra_layers:
+            M = layer.M or wl.M
+            w = (torch.randn((layer.N, layer.K), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+            x = make_device_x(wl, M, layer.K, gen)
+            bias = (torch.randn((layer.N,), generator=gen, device="cuda") * 0.01).to(torch.bfloat16)
+            ax = x.abs().amax(dim=0).double().clamp_min(1e-5).cpu().numpy()
+            aw = w.abs().amax(dim=0).double().clamp_min(1e-5).cpu().numpy()
+            smooth = np.stack([1.0 / (ax ** a / aw ** (1.0 - a)) for a in alphas]).astype(np.float32)
+            signs = (rng.integers(0, 2, (wl.num_groups, layer.K)) * 2 - 1).astype(np.int8)
+            rot = trdq.Rotation(layer.K, wl.t_bounds, signs, smooth)
+            wts = trdq.trdq_prepare_weights(rot, w, wl.wbits)
+            codes = torch.empty((M, layer.K), dtype=torch.int8, device="cuda")
+            scales = torch.empty((M,), dtype=torch.float32, device="cuda")
+            y = torch.empty((M, layer.N), dtype=torch.bfloat16, device="cuda")
+            layers.add(rot, wts, x, codes, scales, bias, y)
+            del w
+    torch.cuda.synchronize()
+    return layers
+
+
+def time_region(fn, steps: int):
+    """CUDA-event time (ms) of `steps` calls of fn(i) on the current stream, synchronised on both sides."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def kernel_pass_ms(layers, wl, which: str, reps: int):
+    """Average time (ms) of one step's launches of ONE kernel kind, replayed from a CUDA graph so the
+    launches are back to back.  which = 'rq' (rotate + quantize) or 'gemm' (GEMM + epilogue)."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    t = int(wl.timesteps()[0])
+    keep = layers._keep
+
+    def issue():
+        for rot, w, x, codes, scales, bias, y in keep:
+            if which == "rq":
+                trdq.trdq_rotate_quantize(rot, t, x, codes, scales)
+            else:
+                trdq.trdq_linear(w, t, codes, scales, bias, y)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        issue()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        issue()
+    for _ in range(3):
+        graph.replay()
+    ms = time_region(lambda i: graph.replay(), reps)
+    return ms / reps
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+def oracle_block_inputs(wl: WL.Workload, rows: int):
+    """Inputs of the linears of ONE transformer block, `rows` tokens each, with the oracle's own
+    (untimed, offline) weight preparation for the first time-step's group."""
+    from oracle import trdq_oracle as O
+    t = int(wl.timesteps()[0])
+    g = O.group_of(wl.t_bounds, t)
+    items = []
+    for li, layer in enumerate(wl.layers + wl.extra_layers):
+        m = min(rows, layer.M or wl.M)
+        inp = WL.make_layer_inputs(wl, li, M=m)
+        act, wv = O.fused_vectors(inp.signs[g], None if inp.smooth is None else inp.smooth[g])
+        if wl.wbits == 8:
+            qw, sw = O.prepare_w8(inp.w, wv)
+        else:
+            qw, sw = O.prepare_w4(inp.w, wv)
+        items.append((inp, act, qw, sw, m))
+    return items
+
+
+def oracle_block_seconds(wl: WL.Workload, items) -> float:
+    """Wall time of the oracle's online path (rotate + quantize, integer GEMM, epilogue) on the block."""
+    from oracle import trdq_oracle as O
+    t0 = time.perf_counter()
+    for inp, act, qw, sw, m in items:
+        q, sx = O.rotate_quantize(inp.x, act)
+        rows = np.arange(m)
+        if wl.wbits == 8:
+            O.linear_w8_rows(q, sx, qw, sw, inp.bias, rows)
+        else:
+            O.linear_w4_rows(q, sx, qw, sw, inp.bias, rows)
+    return time.perf_counter() - t0
+
+
+def block_ops(wl: WL.Workload, rows: int) -> float:
+    return sum(2.0 * min(rows, l.M or wl.M) * l.N * l.K for l in wl.layers + wl.extra_layers)
+
+
+def cpu_baseline(wl: WL.Workload, budget_s: float = 20.0):
+    """The oracle as it stands on this host's cores, on a bounded sample: one block of the step,
+    with as many token rows as fit the time budget (calibrated on 32 rows first)."""
+    from oracle import trdq_oracle as O
+    cal_rows = 32
+    cal = oracle_block_inputs(wl, cal_rows)
+    oracle_block_seconds(wl, cal)                                  # warm the thread pool
+    per_row = oracle_block_seconds(wl, cal) / cal_rows
+    rows = int(max(cal_rows, min(wl.M, budget_s / max(per_row, 1e-9))))
+    items = oracle_block_inputs(wl, rows)
+    sec = oracle_block_seconds(wl, items)
+    tops = block_ops(wl, rows) / sec / 1e12
+    return {"value": tops, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"1 of {wl.blocks} blocks ({len(items)} linears), first {rows} of {wl.M} token rows, {sec:.2f} s"}
+
+
+def run_reference(args, wl: WL.Workload):
+    """`--impl reference`: the CPU oracle on this host, each step a bounded sample of the workload."""
+    from oracle import trdq_oracle as O
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total_steps = args.steps + args.warmup
+    cal_rows = 16
+    cal = oracle_block_inputs(wl, cal_rows)
+    oracle_block_seconds(wl, cal)
+    per_row = oracle_block_seconds(wl, cal) / cal_rows
+    budget = 120.0 / max(total_steps, 1)
+    rows = int(max(8, min(wl.M, budget / max(per_row, 1e-9))))
+    items = oracle_block_inputs(wl, rows)
+    for _ in range(args.warmup):
+        oracle_block_seconds(wl, items)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_block_seconds(wl, items)
+    sec = time.perf_counter() - t0
+    tops = block_ops(wl, rows) * args.steps / sec / 1e12
+    sample = f"each step = 1 of {wl.blocks} blocks, first {rows} of {wl.M} token rows, on host cores"
+    line = {"impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec / max(args.steps, 1) * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": wl.name, "M": wl.M, "blocks": wl.blocks, "sample": sample},
+            "cpu_baseline": {"value": tops, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args, wl: WL.Workload):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_06564_b200 import build as lib_build, trdq
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+    trdq.lib()                                   # fails loudly if the CUDA library is missing
+
+    # weak scaling: every rank runs the whole workload on its own batch (rows are independent; no collective)
+    layers = build_device_workload(wl, seed=1234 + rank, blocks=wl.blocks)
+    ts = wl.timesteps()
+    n_ops = len(layers)
+
+    def step(i):
+        trdq.trdq_run_layers(layers, int(ts[i % len(ts)]))
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    assert trdq.trdq_device_status() == 0
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    if world > 1:
+        dist.barrier()
+    ms = time_region(step, args.steps)
+    if world > 1:
+        tmax = torch.tensor([ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+        dist.barrier()
+    # per-kernel passes (same buffers, launches back to back from a CUDA graph)
+    reps = max(3, min(args.steps, 20))
+    ms_rq = kernel_pass_ms(layers, wl, "rq", reps)
+    ms_gemm = kernel_pass_ms(layers, wl, "gemm", reps)
+    clocks = sampler.stop()
+    assert trdq.trdq_device_status() == 0, "a bounded device-side wait expired during the benchmark"
+
+    ops = step_ops(wl)
+    ms_per_step = ms / args.steps
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    # end to end through the public call with host buffers: H2D of every X, the step, D2H of every Y
+    e2e_steps = max(1, min(args.steps, 3))
+    host_x = [torch.empty(k[2].shape, dtype=k[2].dtype).pin_memory() for k in layers._keep]
+    host_y = [torch.empty(k[6].shape, dtype=k[6].dtype).pin_memory() for k in layers._keep]
+    for hx, k in zip(host_x, layers._keep):
+        hx.copy_(k[2])
+    h2d = sum(h.numel() * h.element_size() for h in host_x)
+    d2h = sum(h.numel() * h.element_size() for h in host_y)
+
+    def e2e_step(i):
+        for hx, k in zip(host_x, layers._keep):
+            k[2].copy_(hx, non_blocking=True)
+        step(i)
+        for hy, k in zip(host_y, layers._keep):
+            hy.copy_(k[6], non_blocking=True)
+
+    e2e_step(0)
+    ms_e2e = time_region(e2e_step, e2e_steps) / e2e_steps
+    if world > 1:
+        tmax = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_e2e = float(tmax.item())
+
+    peaks = load_peaks()
+    in_long_step = True
+    bf16_peak = peaks["bf16_tflops_sustained"] if in_long_step else peaks["bf16_tflops"]
+    int8_peak = bf16_peak * INT8_OVER_BF16
+    gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
+    rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8" if wl.wbits == 8 else "int8xint4", "data": "synthetic",
+        "config": {"workload": wl.name, "M": wl.M, "blocks": wl.blocks, "linears_per_step": n_ops, "groups": wl.num_groups,
+                   "sampling_steps": wl.steps, "wbits": wl.wbits, "parallelism": f"replicas x{world} (rows independent)",
+                   "l2": "inputs larger than L2: every linear has its own X, codes, Y and weights"},
+        "us_per_dit_step": ms_per_step * 1e3,
+        "rotate_quantize_gbs": rq_gbs,
+        "gemm_tops": gemm_tops,
+        "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
+        "roofline": {"kernel": "gemm_w8a8_kernel", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
+                     "unit": "TOPS", "frac": gemm_tops / int8_peak, "traffic": None,
+                     "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
+        "roofline_rotate_quantize": {"kernel": "rotate_quantize_kernel", "bound": "hbm", "achieved": rq_gbs,
+                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
+                                     "traffic": None, "peak_source": peaks["_source"]},
+        "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},
+        "gpu_launches": 2 * n_ops * args.steps,
+        "clocks": clocks,
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, help="index into the workload list (1 = DiT-XL/2 256px, M = 4096)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WL.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -111,6 +111,10 @@ trdq_status trdq_weights_info(const trdq_weights* w, int32_t* N, int32_t* K, int
  * the memory stays owned by `w`. */
 trdq_status trdq_weights_view(const trdq_weights* w, int32_t g, const void** Wq, const float** scales);
 
+/* Copies group g's codes and scales into caller-owned device buffers of exactly the sizes given
+ * in trdq_prepare_weights (device-to-device, asynchronous on `stream`); either may be NULL. */
+trdq_status trdq_weights_export(const trdq_weights* w, int32_t g, void* codes_out, float* scales_out, void* stream);
+
 /* Online activation path G_t(X) followed by dynamic per-token quantization (Sec. 3.1 Eq. 1-2,
  * Sec. 3.2 "calculating quantization parameters online"):
  *   v[m, :]   = (x[m, :] o act_g) . BlockDiag(H_128), fp32 butterflies in the order h = 1, 2, ..., 64
@@ -138,6 +142,27 @@ trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, c
 trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
                             const int32_t M[2], const void* bias_bf16, void* const Y_bf16[2], const int64_t ldy[2],
                             void* stream);
+
+/* One quantized linear layer of a denoising step: rotate + quantize X into the caller's code and
+ * scale buffers, then the integer GEMM with its epilogue into Y (shapes as in the two calls above). */
+typedef struct trdq_layer_op {
+  const trdq_rotation* rot; /* tables for this layer's C_in */
+  const trdq_weights* w;    /* prepared weights; w's K must equal rot's K */
+  const void* X_bf16;       /* dev [M, ldx] */
+  int64_t ldx;
+  int32_t M;
+  int8_t* codes;            /* dev [M, K] scratch owned by the caller */
+  float* scales;            /* dev [M] scratch owned by the caller */
+  const void* bias_bf16;    /* dev [N] or NULL */
+  void* Y_bf16;             /* dev [M, ldy] */
+  int64_t ldy;
+} trdq_layer_op;
+
+/* Runs `count` layer ops in order for time-step t on `stream`: the group switch of the sampling
+ * loop (Sec. 3.2: every layer selects its parameter set by the current time-step) without one
+ * host round trip per kernel.  Validates every op before launching anything.  TRDQ_ERR_MISMATCH
+ * if an op's rot and w disagree in K or in their time-step bounds. */
+trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, void* stream);
 
 /* Raw accumulators of the integer GEMM (wbits = 8 only): acc[m, n] = sum_k q[m,k] * qw_g[n,k],
  * dev int32 [M, ldacc], ldacc >= N, ldacc % 4 == 0.  Exists so that the exact integer result

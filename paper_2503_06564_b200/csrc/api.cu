@@ -240,6 +240,20 @@ trdq_status trdq_weights_view(const trdq_weights* w, int32_t g, const void** Wq,
   return TRDQ_OK;
 }
 
+trdq_status trdq_weights_export(const trdq_weights* w, int32_t g, void* codes_out, float* scales_out, void* stream) {
+  if (!w) return TRDQ_ERR_NULL;
+  if (g < 0 || g >= w->num_groups) return TRDQ_ERR_GROUP;
+  const size_t code_bytes = w->wbits == 8 ? static_cast<size_t>(w->N) * w->K : static_cast<size_t>(w->N) * w->K / 2;
+  const size_t scale_count = w->wbits == 8 ? static_cast<size_t>(w->N) : static_cast<size_t>(w->N) * (w->K / TRDQ_BLOCK);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (codes_out && cudaMemcpyAsync(codes_out, w->groups[g].codes, code_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return TRDQ_ERR_CUDA;
+  if (scales_out &&
+      cudaMemcpyAsync(scales_out, w->groups[g].scales, scale_count * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return TRDQ_ERR_CUDA;
+  return TRDQ_OK;
+}
+
 trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, int8_t* codes,
                                  float* scales, void* stream) {
   if (!rot) return TRDQ_ERR_NULL;
@@ -299,6 +313,30 @@ trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes,
   void* y[2] = {acc, nullptr};
   const int64_t l[2] = {ldacc, ldacc};
   return linear_common(w, t, c, nullptr, m, nullptr, y, l, true, stream);
+}
+
+trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, void* stream) {
+  if (count < 0) return TRDQ_ERR_SHAPE;
+  if (count == 0) return TRDQ_OK;
+  if (!ops) return TRDQ_ERR_NULL;
+  for (int i = 0; i < count; ++i) {
+    const trdq_layer_op& op = ops[i];
+    if (!op.rot || !op.w) return TRDQ_ERR_NULL;
+    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds) return TRDQ_ERR_MISMATCH;
+    if (find_group(op.rot->t_bounds, t) < 0) return TRDQ_ERR_TIMESTEP;
+    if (op.M < 0 || op.ldx < op.rot->K || op.ldy < op.w->N) return TRDQ_ERR_SHAPE;
+    if (op.M > 0 && (!op.X_bf16 || !op.codes || !op.scales || !op.Y_bf16)) return TRDQ_ERR_NULL;
+    if (op.ldx % 8 != 0 || op.ldy % 8 != 0 || !aligned16(op.X_bf16) || !aligned16(op.codes) || !aligned16(op.Y_bf16))
+      return TRDQ_ERR_ALIGN;
+  }
+  for (int i = 0; i < count; ++i) {
+    const trdq_layer_op& op = ops[i];
+    trdq_status st = trdq_rotate_quantize(op.rot, t, op.X_bf16, op.ldx, op.M, op.codes, op.scales, stream);
+    if (st != TRDQ_OK) return st;
+    st = trdq_linear(op.w, t, op.codes, op.scales, op.M, op.bias_bf16, op.Y_bf16, op.ldy, stream);
+    if (st != TRDQ_OK) return st;
+  }
+  return TRDQ_OK;
 }
 
 trdq_status trdq_device_status(uint32_t* word) {

@@ -1,0 +1,75 @@
+"""Single-kernel micro-benchmark: times one kernel of the library on one shape with CUDA events.
+
+    python -m paper_2503_06564_b200.microbench rq   --M 65536 --K 1152
+    python -m paper_2503_06564_b200.microbench gemm --M 16384 --K 1152 --N 4608
+
+Also the small, self-ending command to put under a profiler (few launches, a few hundred MB).
+Buffers are rotated through `--sets` distinct copies so that consecutive launches do not find
+their inputs in L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+
+
+def main():
+    import torch
+    from paper_2503_06564_b200 import build, trdq
+    ap = argparse.ArgumentParser()
+    ap.add_argument("kernel", choices=["rq", "gemm"])
+    ap.add_argument("--M", type=int, default=16384)
+    ap.add_argument("--K", type=int, default=1152)
+    ap.add_argument("--N", type=int, default=4608)
+    ap.add_argument("--wbits", type=int, default=8)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--sets", type=int, default=4)
+    args = ap.parse_args()
+    build.build()
+    torch.manual_seed(0)
+    M, K, N = args.M, args.K, args.N
+    rng = np.random.default_rng(0)
+    signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs, None)
+    xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(args.sets)]
+    codes = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(args.sets)]
+    scales = [torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(args.sets)]
+    if args.kernel == "rq":
+        def run(i):
+            s = i % args.sets
+            trdq.trdq_rotate_quantize(rot, 0, xs[s], codes[s], scales[s])
+        work, unit = M * (3.0 * K + 4.0) / 1e9, "GB/s"
+    else:
+        w = (torch.randn((N, K), device="cuda") * 0.02).to(torch.bfloat16)
+        wts = trdq.trdq_prepare_weights(rot, w, args.wbits)
+        bias = torch.zeros((N,), dtype=torch.bfloat16, device="cuda")
+        ys = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(args.sets)]
+        for s in range(args.sets):
+            trdq.trdq_rotate_quantize(rot, 0, xs[s], codes[s], scales[s])
+
+        def run(i):
+            s = i % args.sets
+            trdq.trdq_linear(wts, 0, codes[s], scales[s], bias, ys[s])
+        work, unit = 2.0 * M * N * K / 1e12, "TOPS"
+    for i in range(args.warmup):
+        run(i)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.iters + 1)]
+    ev[0].record()
+    for i in range(args.iters):
+        run(i)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.iters))
+    med = ms[len(ms) // 2]
+    assert trdq.trdq_device_status() == 0
+    print(json.dumps({"kernel": args.kernel, "M": M, "K": K, "N": N if args.kernel == "gemm" else None, "wbits": args.wbits,
+                      "ms_median": med, "ms_min": ms[0], "rate_median": work / (med * 1e-3), "rate_best": work / (ms[0] * 1e-3),
+                      "unit": unit}))
+
+
+if __name__ == "__main__":
+    main()

@@ -25,7 +25,9 @@ STATUS_NAMES = {0: "TRDQ_OK", 1: "TRDQ_ERR_NULL", 2: "TRDQ_ERR_SHAPE", 3: "TRDQ_
 EXPORTS = (
     "trdq_status_string", "trdq_version", "trdq_rotation_create", "trdq_rotation_destroy", "trdq_group_of",
     "trdq_find_group", "trdq_prepare_weights", "trdq_weights_destroy", "trdq_weights_info", "trdq_weights_view",
+    "trdq_weights_export",
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
+    "trdq_run_layers",
 )
 
 
@@ -38,6 +40,12 @@ class TrdqError(RuntimeError):
 class RotationSpec(C.Structure):
     _fields_ = [("K", C.c_int32), ("block", C.c_int32), ("num_groups", C.c_int32),
                 ("t_bounds", C.POINTER(C.c_int32)), ("signs", C.POINTER(C.c_int8)), ("smooth", C.POINTER(C.c_float))]
+
+
+class LayerOp(C.Structure):
+    _fields_ = [("rot", C.c_void_p), ("w", C.c_void_p), ("X_bf16", C.c_void_p), ("ldx", C.c_int64), ("M", C.c_int32),
+                ("codes", C.c_void_p), ("scales", C.c_void_p), ("bias_bf16", C.c_void_p), ("Y_bf16", C.c_void_p),
+                ("ldy", C.c_int64)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -62,11 +70,13 @@ def lib() -> C.CDLL:
         l.trdq_weights_destroy.argtypes = [vp]
         l.trdq_weights_info.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
         l.trdq_weights_view.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp)]
+        l.trdq_weights_export.argtypes = [vp, i32, vp, vp, vp]
         l.trdq_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp]
         l.trdq_linear.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_linear_cfg.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), vp, C.POINTER(vp),
                                       C.POINTER(i64), vp]
         l.trdq_gemm_i32.argtypes = [vp, i32, vp, i32, vp, i64, vp]
+        l.trdq_run_layers.argtypes = [C.POINTER(LayerOp), i32, i32, vp]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -147,19 +157,13 @@ class Weights:
     def view_tensors(self, g: int):
         """Copies of group g's codes and scales as torch tensors (device)."""
         import torch
-        wq, sc = self.view(g)
         if self.wbits == 8:
             codes = torch.empty((self.N, self.K), dtype=torch.int8, device="cuda")
             scales = torch.empty((self.N,), dtype=torch.float32, device="cuda")
         else:
             codes = torch.empty((self.N, self.K // 2), dtype=torch.uint8, device="cuda")
             scales = torch.empty((self.N, self.K // 128), dtype=torch.float32, device="cuda")
-        cudart = torch.cuda.cudart()
-        torch.cuda.current_stream().synchronize()
-        for dst, src in ((codes, wq), (scales, sc)):
-            err = cudart.cudaMemcpy(dst.data_ptr(), src, dst.numel() * dst.element_size(), 3)  # device -> device
-            if int(err) != 0:
-                raise RuntimeError(f"cudaMemcpy failed: {err}")
+        _check(lib().trdq_weights_export(self._h, int(g), _ptr(codes), _ptr(scales), _stream()), "trdq_weights_export")
         return codes, scales
 
     def close(self) -> None:
@@ -234,6 +238,40 @@ def trdq_gemm_i32(w: Weights, t: int, codes, out=None):
     ld = int(out.stride(0)) if M > 1 else w.N
     _check(lib().trdq_gemm_i32(w._h, int(t), _ptr(codes), M, _ptr(out), ld, _stream()), "trdq_gemm_i32")
     return out
+
+
+class LayerList:
+    """A fixed list of trdq_layer_op records (one denoising step's quantized linears).  Holds
+    references to every tensor and handle it points to."""
+
+    def __init__(self):
+        self._keep = []
+        self._ops = []
+        self._array = None
+
+    def add(self, rot: Rotation, w: Weights, X_bf16, codes, scales, bias_bf16, Y_bf16) -> None:
+        M = int(X_bf16.shape[0])
+        assert X_bf16.stride(1) == 1 and Y_bf16.stride(1) == 1 and codes.is_contiguous()
+        self._ops.append(LayerOp(rot._h, w._h, _ptr(X_bf16), int(X_bf16.stride(0)) if M > 1 else rot.K, M, _ptr(codes),
+                                 _ptr(scales), _ptr(bias_bf16), _ptr(Y_bf16), int(Y_bf16.stride(0)) if M > 1 else w.N))
+        self._keep.append((rot, w, X_bf16, codes, scales, bias_bf16, Y_bf16))
+        self._array = None
+
+    def __len__(self) -> int:
+        return len(self._ops)
+
+    def array(self):
+        if self._array is None:
+            self._array = (LayerOp * len(self._ops))(*self._ops)
+        return self._array
+
+
+def trdq_run_layers(layers: LayerList, t: int, first: int = 0, count: Optional[int] = None) -> None:
+    """All (or a slice of) the layer ops at time-step t on the current stream."""
+    n = len(layers) - first if count is None else count
+    arr = layers.array()
+    ptr = C.cast(C.byref(arr, first * C.sizeof(LayerOp)), C.POINTER(LayerOp))
+    _check(lib().trdq_run_layers(ptr, int(n), int(t), _stream()), "trdq_run_layers")
 
 
 def trdq_device_status() -> int:

@@ -45,6 +45,10 @@ def check_output(y_gpu: np.ndarray, y_ref: np.ndarray, max_ulp: float = 2.0, rel
     err = np.abs(y_gpu - y_ref64)
     ulps = err / bf16_ulp(y_ref)
     l2 = np.sqrt((err ** 2).sum()) / max(np.sqrt((y_ref64 ** 2).sum()), 1e-30)
+    # Rounding to bf16 alone gives a relative L2 error near 1.5e-3 on many samples; on a handful of
+    # outputs the sample fluctuates up to the worst case 2^-8, so the 2e-3 rule needs a real sample.
+    if y_ref.size < 4096:
+        rel_l2 = max(rel_l2, 2.0 ** -8)
     assert l2 <= rel_l2, f"relative L2 error {l2:.3e} > {rel_l2}"
     assert ulps.max() <= max_ulp, f"max error {ulps.max():.3f} bf16 ulp at {np.unravel_index(ulps.argmax(), ulps.shape)}"
     return float(l2), float(ulps.max())
