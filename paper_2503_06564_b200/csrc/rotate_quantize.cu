@@ -185,6 +185,174 @@ __global__ void __launch_bounds__(1024) rotate_quantize_kernel(const __nv_bfloat
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Fast path for per-row int8 codes (the online activation kernel).
+//
+// Four lanes own one 128-block of one row, 32 elements each, as four 16-byte chunks interleaved
+// across the lanes: lane l holds chunks l, l+4, l+8, l+12 (chunk = 8 consecutive elements), so a
+// warp-wide 16-byte load covers whole 32-byte sectors.  With element index bits i0..i6: i0..i2 lie
+// inside a chunk, i3 i4 select the lane, i5 i6 the chunk of a lane.  Stages h = 1, 2, 4, 32, 64 pair
+// registers of a thread, h = 8, 16 pair lanes by shuffle; the stage order h = 1 .. 64 is kept.
+// Values are held as fp32 pairs (i0 = 0, 1) and processed with the packed fp32x2 add / mul / fma
+// instructions of sm_100, each lane of which rounds exactly like the scalar instruction.
+// Rounding to the integer code uses the exact identity rne(y) = (y + 1.5 * 2^23) - 1.5 * 2^23 for
+// |y| < 2^22: after the addition the low byte of the fp32 pattern is the two's-complement code.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFastLanes = 4;
+constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23
+
+__device__ __forceinline__ float2 shfl_xor2(float2 v, int mask) {
+  return make_float2(__shfl_xor_sync(0xffffffffu, v.x, mask), __shfl_xor_sync(0xffffffffu, v.y, mask));
+}
+
+__device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
+  const uint32_t lo = __byte_perm(__float_as_uint(a.x), __float_as_uint(a.y), 0x0040);
+  const uint32_t hi = __byte_perm(__float_as_uint(b.x), __float_as_uint(b.y), 0x0040);
+  return __byte_perm(lo, hi, 0x5410);
+}
+
+template <int MIN_CTAS>
+__global__ void __launch_bounds__(320, MIN_CTAS)
+rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K, const float* __restrict__ vec,
+                            int8_t* __restrict__ codes, float* __restrict__ scales, int32_t rows_per_tile, float zero) {
+  extern __shared__ float svec[];  // the group's fused vector, K floats
+  __shared__ unsigned int row_max[3][32];
+  const int nb = K / TRDQ_BLOCK;
+  const int lane4 = threadIdx.x & (kFastLanes - 1);
+  const int item = threadIdx.x / kFastLanes;
+  const bool active = item < rows_per_tile * nb;
+  const int r = active ? item / nb : 0;
+  const int b = active ? item % nb : 0;
+
+  for (int i = threadIdx.x; i < K / 4; i += blockDim.x) reinterpret_cast<float4*>(svec)[i] = __ldg(reinterpret_cast<const float4*>(vec) + i);
+  if (threadIdx.x < 32) row_max[0][threadIdx.x] = 0u;
+  __syncthreads();
+
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  const int col0 = b * TRDQ_BLOCK + lane4 * 8;  // first element of chunk 0 of this lane; chunk c is 32 further
+  const float2* sv = reinterpret_cast<const float2*>(svec + col0);
+
+  uint4 raw[4];
+  auto fetch = [&](int tile) {
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    if (active && tile < num_tiles && row < M) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + col0);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) raw[c] = __ldg(src + 4 * c);  // +32 elements = +4 uint4
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) raw[c] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  fetch(blockIdx.x);
+
+  int it = 0;
+  for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    const int buf = it % 3;
+    if (threadIdx.x < 32) row_max[(it + 1) % 3][threadIdx.x] = 0u;
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    const bool valid = active && row < M;
+
+    // v[4c + j] = elements (2j, 2j+1) of chunk c, scaled by the fused vector
+    float2 v[16];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 xv = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+        v[4 * c + j] = __fmul2_rn(xv, sv[16 * c + j]);
+      }
+    }
+    fetch(tile + gridDim.x);  // next tile's rows are in flight while this one is transformed
+
+    // h = 1: inside a pair
+#pragma unroll
+    for (int p = 0; p < 16; ++p) v[p] = make_float2(__fadd_rn(v[p].x, v[p].y), __fsub_rn(v[p].x, v[p].y));
+    // h = 2, 4: pair index bits 0, 1
+#pragma unroll
+    for (int hb = 1; hb <= 2; hb <<= 1) {
+#pragma unroll
+      for (int p = 0; p < 16; ++p) {
+        if ((p & hb) == 0) {
+          const float2 a = v[p], c2 = v[p + hb];
+          v[p] = __fadd2_rn(a, c2);
+          v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+        }
+      }
+    }
+    // h = 8, 16: lanes l ^ 1, l ^ 2; upper lane computes other - own, lower lane own + other
+#pragma unroll
+    for (int mask = 1; mask <= 2; mask <<= 1) {
+      const float sgn = (lane4 & mask) ? -1.0f : 1.0f;
+      const float2 s2 = make_float2(sgn, sgn);
+#pragma unroll
+      for (int p = 0; p < 16; ++p) v[p] = __ffma2_rn(v[p], s2, shfl_xor2(v[p], mask));
+    }
+    // h = 32, 64: pair index bits 2, 3 (the chunk of the lane)
+#pragma unroll
+    for (int hb = 4; hb <= 8; hb <<= 1) {
+#pragma unroll
+      for (int p = 0; p < 16; ++p) {
+        if ((p & hb) == 0) {
+          const float2 a = v[p], c2 = v[p + hb];
+          v[p] = __fadd2_rn(a, c2);
+          v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+        }
+      }
+    }
+
+    float m = 0.0f;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    if (valid && lane4 == 0) atomicMax(&row_max[buf][r], __float_as_uint(m));
+    __syncthreads();
+
+    if (valid) {
+      const float amax = __uint_as_float(row_max[buf][r]);
+      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+      const float2 inv2 = make_float2(inv, inv);
+      const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
+      // The product must be rounded to fp32 before the magic addition rounds it to an integer.  A packed
+      // multiply feeding a packed add gets contracted into one fused operation (a single rounding) by
+      // the assembler, so the product is written as fma(v, inv, zero) with `zero` a kernel argument
+      // equal to 0.0f: one rounding of v * inv, and nothing left to contract.
+      const float2 zero2 = make_float2(zero, zero);
+      int8_t* dst = codes + row * K + col0;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float2 q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
+        *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
+      }
+      if (b == 0 && lane4 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
+    }
+  }
+}
+
+cudaError_t launch_rows_fast(const void* x, int64_t ldx, int32_t M, int32_t K, const float* vec, void* codes, float* scales,
+                             cudaStream_t stream) {
+  const int nb = K / TRDQ_BLOCK;
+  int rows = 72 / nb;  // about 72 lane groups (288 threads) per CTA
+  if (rows < 1) rows = 1;
+  if (rows > 32) rows = 32;
+  int threads = rows * nb * kFastLanes;
+  threads = (threads + 31) / 32 * 32;
+  const int num_tiles = (M + rows - 1) / rows;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = min(num_tiles, sms * 2);
+  const size_t smem = static_cast<size_t>(K) * sizeof(float);
+  rotate_quantize_rows_kernel<2><<<grid, threads, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), ldx, M, K, vec,
+                                                                  static_cast<int8_t*>(codes), scales, rows, 0.0f);
+  return cudaGetLastError();
+}
+
 template <int MODE, int P>
 cudaError_t launch(const void* x, int64_t ldx, int32_t M, int32_t K, const float* vec, void* codes, float* scales,
                    int rows_per_tile, int groups, cudaStream_t stream) {
@@ -224,7 +392,12 @@ cudaError_t dispatch(const void* x, int64_t ldx, int32_t M, int32_t K, const flo
 cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
                                    void* codes, float* scales, cudaStream_t stream) {
   if (M == 0) return cudaSuccess;
-  if (mode == 0) return dispatch<0>(x_bf16, ldx, M, K, vec, codes, scales, stream);
+  if (mode == 0) {
+    // fast path: the whole tile of a CTA fits 320 threads and the vector fits the default shared memory
+    if (K / TRDQ_BLOCK <= 80 && static_cast<size_t>(K) * sizeof(float) <= 40 * 1024)
+      return launch_rows_fast(x_bf16, ldx, M, K, vec, codes, scales, stream);
+    return dispatch<0>(x_bf16, ldx, M, K, vec, codes, scales, stream);
+  }
   return dispatch<1>(x_bf16, ldx, M, K, vec, codes, scales, stream);
 }
 
