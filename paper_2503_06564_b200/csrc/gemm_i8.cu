@@ -7,8 +7,11 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction,
 //               four per stage); accumulators live in tensor memory, two stages of BN columns
 //   warp 2      allocates / frees tensor memory
-//   warps 4-7   epilogue: tcgen05.ld of the finished accumulator (warp q reads lanes 32q..32q+31,
-//               one output row per thread), fp32 dequantization, bf16 pack, 16-byte stores
+//   warps 4-11  epilogue: tcgen05.ld of the finished accumulator (a warp reads the tensor-memory
+//               lanes 32*(warp%4) .. +31, one output row per thread; warps 4-7 take the left half of
+//               the columns, warps 8-11 the right half), fp32 dequantization, bf16 pack into a
+//               swizzled 32 x 32 staging tile in shared memory, one TMA store per tile of 32 columns
+//               (row-scattered 16-byte stores from registers turned out to bound the whole kernel)
 // The epilogue of tile i overlaps the main loop of tile i+1 through the second accumulator.
 // Tiles are visited column-block major so that concurrently running CTAs share one weight
 // tile; both CFG row segments are part of the same tile list, so a weight tile is fetched
@@ -24,8 +27,8 @@ namespace {
 constexpr int kTileM = 128;
 constexpr int kTileKBytes = 128;  // one swizzle atom: 128 int8 along K per stage
 constexpr int kUmmaK = 32;        // K of one kind::i8 instruction
-constexpr int kThreads = 256;
-constexpr int kEpilogueThreads = 128;
+constexpr int kThreads = 384;
+constexpr int kEpilogueThreads = 256;
 constexpr int kAccStride = 256;   // tensor-memory columns between the two accumulator stages
 constexpr int kTmemCols = 512;
 constexpr int kSmemBudget = 227 * 1024;
@@ -35,11 +38,14 @@ struct Cfg {
   static constexpr int kABytes = kTileM * kTileKBytes;
   static constexpr int kBBytes = BN * kTileKBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  // parameters staged for the epilogue: (sw, bias) per column, one buffer per accumulator stage
-  static constexpr int kParamBytes = 2 * BN * 8;
+  // parameters staged for the epilogue: (sw, bias) and the cancellation threshold per column, one
+  // buffer per accumulator stage
+  static constexpr int kParamBytes = 2 * BN * 12;
   static constexpr int kBarrierBytes = 256;
-  static constexpr int kStages = (kSmemBudget - 1024 - kParamBytes - kBarrierBytes) / kStageBytes;
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kParamBytes + kBarrierBytes;
+  // output staging: one 32-row x 32-column bf16 tile (2 KB, 64-byte swizzle) per epilogue warp
+  static constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 2048;
+  static constexpr int kStages = (kSmemBudget - 1024 - kOutStageBytes - kParamBytes - kBarrierBytes) / kStageBytes;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes;
   static_assert(kStages >= 3, "pipeline too shallow");
   static_assert(kStages <= 12, "barrier area too small");
 };
@@ -47,6 +53,7 @@ struct Cfg {
 struct alignas(64) GemmParams {
   CUtensorMap tmap_a[2];
   CUtensorMap tmap_b;
+  CUtensorMap tmap_out[2];  // bf16 output of each segment, box 32 x 32, 64-byte swizzle
   const float* sx[2];
   void* out[2];
   int64_t ld[2];
@@ -80,8 +87,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
-  float2* param_buf = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes + C::kParamBytes);
+  const uint32_t out_stage_base = smem_base + C::kStages * C::kStageBytes;
+  float2* param_buf = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes + C::kOutStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes + C::kOutStageBytes + C::kParamBytes);
   // barrier layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then the tensor-memory base address
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8 * C::kStages;
@@ -120,6 +128,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
       prefetch_tensormap(&p.tmap_a[0]);
       prefetch_tensormap(&p.tmap_a[1]);
       prefetch_tensormap(&p.tmap_b);
+      prefetch_tensormap(&p.tmap_out[0]);
+      prefetch_tensormap(&p.tmap_out[1]);
       BoundedWaiter w(p.status, kStatusTimeoutProducer);
       int stage = 0;
       uint32_t phase = 0;
@@ -180,14 +190,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
     }
   } else if (warp >= 4) {
     // ---------------------------------------------------------------- epilogue
-    const int q = warp - 4;                 // lane quarter of tensor memory this warp may read
-    const int et = threadIdx.x - 4 * 32;    // 0..127
+    const int ew = warp - 4;                // 0..7
+    const int q = ew & 3;                   // = warp % 4: the lane quarter of tensor memory this warp may read
+    const int half = ew >> 2;               // which half of the tile's columns
+    const int et = threadIdx.x - 4 * 32;    // 0..255
+    constexpr int kChunksPerWarp = BN / 64; // 32-column chunks per warp
+    const uint32_t my_stage = out_stage_base + ew * 2048;
     BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const TileCoord tc = tile_coord(p, tile, BN);
-      float2* pb = param_buf + acc * BN;
+      float2* pb = param_buf + acc * BN;                                           // (sw, bias)
+      float* thr = reinterpret_cast<float*>(param_buf + 2 * BN) + acc * BN;        // 2^-10 * |bias|
       if (MODE == 0) {
         for (int c = et; c < BN; c += kEpilogueThreads) {
           const int n = tc.n0 + c;
@@ -197,6 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
             v.y = p.bias ? __bfloat162float(p.bias[n]) : 0.0f;
           }
           pb[c] = v;
+          thr[c] = fabsf(v.y) * 0.0009765625f;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
       }
@@ -209,40 +225,59 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccStride;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc = 0; cc < kChunksPerWarp; ++cc) {
+        const int c = half * kChunksPerWarp + cc;
         uint32_t r[32];
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
         const int n_base = tc.n0 + c * 32;
-        if (!row_ok) continue;
         if (MODE == 0) {
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out[tc.seg]) + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
+          const float4* pb4 = reinterpret_cast<const float4*>(pb + c * 32);
+          const float4* thr4 = reinterpret_cast<const float4*>(thr + c * 32);
           uint32_t packed[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float y[2];
+          for (int j = 0; j < 32; j += 4) {
+            const float4 p01 = pb4[j / 2], p23 = pb4[j / 2 + 1], th = thr4[j / 4];
+            const float swv[4] = {p01.x, p01.z, p23.x, p23.z};
+            const float bv[4] = {p01.y, p01.w, p23.y, p23.w};
+            const float tv[4] = {th.x, th.y, th.z, th.w};
+            float y[4];
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const float2 sb = pb[c * 32 + j + e];
+            for (int e = 0; e < 4; ++e) {
               const int32_t a = static_cast<int32_t>(r[j + e]);
               const float af = static_cast<float>(a);
-              // sx*sw as an unevaluated sum s_hi + s_lo (exact), so that a cancellation between
-              // the product and the bias does not expose the rounding of the scale product
-              const float s_hi = __fmul_rn(sxm, sb.x);
-              const float s_lo = __fmaf_rn(sxm, sb.x, -s_hi);
-              float v = __fmaf_rn(af, s_lo, __fmaf_rn(af, s_hi, sb.y));
-              if (fabsf(af) >= 16777216.0f) v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
+              const float s_hi = __fmul_rn(sxm, swv[e]);
+              float v = __fmaf_rn(af, s_hi, bv[e]);
+              // fp32 is accurate to 2^-23 of the product.  Only when product and bias cancel to less
+              // than 2^-10 of the bias can that exceed a bf16 rounding step of the result; then the
+              // scale product is carried as an exact two-term sum and the part of the accumulator
+              // that fp32 could not hold is added back.
+              if (fabsf(v) < tv[e]) {
+                const float s_lo = __fmaf_rn(sxm, swv[e], -s_hi);
+                v = __fmaf_rn(af, s_lo, v);
+                v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
+              }
               y[e] = v;
             }
-            const __nv_bfloat162 h = __floats2bfloat162_rn(y[0], y[1]);
-            packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]);
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2], y[3]);
+            packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h0);
+            packed[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h1);
           }
+          // staging tile: row = lane, 64 bytes per row, 16-byte chunk j stored at j ^ ((lane >> 1) & 3)
+          if (lane == 0) bulk_wait_group_read<0>();  // the previous store has finished reading the tile
+          __syncwarp();
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (n_base + 8 * v < p.N)
-              *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+          for (int v = 0; v < 4; ++v)
+            st_shared_v4(my_stage + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4), packed[4 * v], packed[4 * v + 1], packed[4 * v + 2],
+                         packed[4 * v + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&p.tmap_out[tc.seg], n_base, tc.m0 + q * 32, my_stage);  // rows >= M and columns >= N are clipped
+            bulk_commit_group();
           }
-        } else {
+        } else if (row_ok) {
           int32_t* out = static_cast<int32_t*>(p.out[tc.seg]) + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
@@ -259,6 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
         acc_phase ^= 1;
       }
     }
+    if (MODE == 0 && lane == 0) bulk_wait_group<0>();  // every output tile has been written
     w.settle();
   }
 
@@ -331,6 +367,13 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
                                           static_cast<uint64_t>(w->K), kTileKBytes, kTileM);
     if (st != TRDQ_OK) return st;
   }
+  for (int s = 0; s < 2 && !raw_i32; ++s) {
+    const GemmSegment& src = seg[s].M > 0 ? seg[s] : seg[1 - s];
+    trdq_status st = encode_tmap_2d(&p.tmap_out[s], src.out, 2, static_cast<uint64_t>(w->N), static_cast<uint64_t>(src.M),
+                                    static_cast<uint64_t>(src.ld) * 2, 32, 32, 64);
+    if (st != TRDQ_OK) return st;
+  }
+  if (raw_i32) p.tmap_out[0] = p.tmap_out[1] = p.tmap_a[0];  // unused by the raw-accumulator mode
   p.tmap_b = w->groups[g].tmap_b[ti];
   p.sw = w->groups[g].scales;
   p.bias = static_cast<const __nv_bfloat16*>(bias_bf16);

@@ -64,5 +64,9 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
 // 2-D uint8 row-major [rows, row_bytes-wide], box = 128 bytes x box_rows, 128-byte swizzle.
 trdq_status encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
                                  uint64_t row_stride_bytes, uint32_t box_bytes, uint32_t box_rows);
+// General 2-D row-major map: `cols` elements of `elem_bytes` (1, 2 or 4) per row, box = box_cols x box_rows,
+// swizzle_bytes in {0, 32, 64, 128}.
+trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint64_t cols, uint64_t rows,
+                           uint64_t row_stride_bytes, uint32_t box_cols, uint32_t box_rows, uint32_t swizzle_bytes);
 
 }  // namespace trdq
