@@ -221,11 +221,26 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
       return TRDQ_ERR_CUDA;
     }
     for (int i = 0; i < kNumTileN; ++i) {
-      const uint32_t box_rows = wbits == 8 ? kTileN[i] : 128;
-      const trdq_status st = encode_tmap_u8_sw128(&gw.tmap_b[i], gw.codes, row_bytes, N, row_bytes, box_bytes, box_rows);
+      const trdq_status st = wbits == 8
+                                 ? encode_tmap_u8_sw128(&gw.tmap_b[i], gw.codes, row_bytes, N, row_bytes, box_bytes, kTileN[i])
+                                 : encode_tmap_2d(&gw.tmap_b[i], gw.codes, 1, row_bytes, N, row_bytes, box_bytes, 128, 0);
       if (st != TRDQ_OK) {
         trdq_weights_destroy(w);
         return st;
+      }
+    }
+    if (wbits == 4) {
+      const int n_pad = (N + 127) / 128 * 128;
+      const int groups = K / TRDQ_BLOCK;
+      if (cudaMalloc(&gw.mult_t, static_cast<size_t>(groups) * n_pad * sizeof(int32_t)) != cudaSuccess ||
+          cudaMalloc(&gw.base, static_cast<size_t>(n_pad) * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_NOMEM;
+      }
+      if (launch_w4_multipliers(gw.scales, N, groups, n_pad, gw.mult_t, gw.base, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_CUDA;
       }
     }
   }
@@ -238,6 +253,8 @@ trdq_status trdq_weights_destroy(trdq_weights* w) {
   for (auto& gw : w->groups) {
     if (gw.codes) cudaFree(gw.codes);
     if (gw.scales) cudaFree(gw.scales);
+    if (gw.mult_t) cudaFree(gw.mult_t);
+    if (gw.base) cudaFree(gw.base);
   }
   delete w;
   return TRDQ_OK;

@@ -26,7 +26,11 @@ constexpr int kTileN[kNumTileN] = {128, 192, 256};
 struct GroupWeights {
   void* codes = nullptr;                // dev int8 [N,K] or packed uint8 [N,K/2]
   float* scales = nullptr;              // dev fp32 [N] or [N,K/128]
-  CUtensorMap tmap_b[kNumTileN];        // TMA descriptors of `codes`, one per tile width
+  CUtensorMap tmap_b[kNumTileN];        // TMA descriptors of `codes`, one per tile width (4-bit: only [0], 128 rows x 64 bytes)
+  // 4-bit weights only: the scales of an output channel as integers on a common power-of-two grid,
+  //   scales[n][kg] = mult_t[kg][n] * base[n]   (exact whenever the exponents of a channel span < 7 bits)
+  int32_t* mult_t = nullptr;            // dev int32 [K/128][n_pad], n_pad = N rounded up to 128
+  float* base = nullptr;                // dev fp32 [n_pad], a power of two (already divided by 16, see gemm_w4a8.cu)
 };
 
 }  // namespace trdq
@@ -59,6 +63,8 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
                            cudaStream_t stream);
 trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
                            cudaStream_t stream);
+cudaError_t launch_w4_multipliers(const float* scales, int32_t N, int32_t groups, int32_t n_pad, int32_t* mult_t, float* base,
+                                  cudaStream_t stream);
 
 // tensor maps (driver entry point fetched through the runtime; no link-time libcuda dependency)
 // 2-D uint8 row-major [rows, row_bytes-wide], box = 128 bytes x box_rows, 128-byte swizzle.

@@ -180,3 +180,57 @@ def test_linear_strided_output_and_cfg_segments():
         trdq.trdq_linear(wts, t, codes, scales, bias_d, out=torch.empty((M, N + 4), dtype=torch.bfloat16, device="cuda")[:, :N])
     assert e.value.status == 3
     assert trdq.trdq_device_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K,with_bias", [
+    (300, 1152, 1152, True),     # 9 scale groups, ragged rows
+    (129, 1168, 4608, True),     # 36 groups: accumulators rotate many times; N is not a multiple of the tile
+    (1, 16, 128, False),         # one group, smallest problem
+    (260, 3456, 1152, False),
+])
+def test_linear_w4a8_matches_oracle(M, N, K, with_bias):
+    """int4 weights with one scale per (channel, 128 k): per-group integer sums, scaled and added."""
+    from paper_2503_06564_b200 import trdq
+    G = 2
+    rot, wts, bounds, bias, ref = _setup(N, K, G, 400 + N + K, wbits=4)
+    assert wts.wbits == 4
+    x = _acts(M, K, 27 + M)
+    xd = to_dev_bf16(x)
+    bias_d = to_dev_bf16(bias) if with_bias else None
+    for g in range(G):
+        t = int(bounds[g])
+        act, packed_ref, sw4_ref = ref[g]
+        packed_dev, sw4_dev = wts.view_tensors(g)
+        assert np.array_equal(packed_dev.cpu().numpy(), packed_ref) and np.array_equal(sw4_dev.cpu().numpy(), sw4_ref)
+        q_ref, sx_ref = O.rotate_quantize(x, act)
+        codes, scales = trdq.trdq_rotate_quantize(rot, t, xd)
+        assert np.array_equal(codes.cpu().numpy(), q_ref)
+        y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
+        y_ref = O.linear_w4_rows(q_ref, sx_ref, packed_ref, sw4_ref, bias if with_bias else None, np.arange(M))
+        l2, ulps = check_output(bf16_to_f32_np(y), y_ref, max_ulp=2.0, rel_l2=2e-3)
+        assert ulps <= 1.0
+    assert trdq.trdq_device_status() == 0
+
+
+def test_linear_w4a8_group_scales_of_very_different_size():
+    """Channels whose group scales span many binades (one huge weight in one block): the common-grid
+    integer multipliers lose low bits of the small scales only, far below a bf16 step of the result."""
+    from paper_2503_06564_b200 import trdq
+    M, N, K = 140, 128, 1024
+    rng = np.random.default_rng(77)
+    signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs, None)
+    w = rng.standard_normal((N, K)) * 0.02
+    w[:, 0:128] *= 3000.0          # group 0 is 3000 x larger than the others
+    w[5, 256:384] = 0.0            # an all-zero group: scale 0, codes 0
+    wb = WL.to_bf16_bits(w)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(wb), 4)
+    act, wv = O.fused_vectors(signs[0], None)
+    packed_ref, sw4_ref = O.prepare_w4(wb, wv)
+    assert sw4_ref[5, 2] == 0.0
+    x = _acts(M, K, 5)
+    q_ref, sx_ref = O.rotate_quantize(x, act)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, to_dev_bf16(x))
+    y = trdq.trdq_linear(wts, 0, codes, scales, None)
+    y_ref = O.linear_w4_rows(q_ref, sx_ref, packed_ref, sw4_ref, None, np.arange(M))
+    check_output(bf16_to_f32_np(y), y_ref, max_ulp=1.0)
