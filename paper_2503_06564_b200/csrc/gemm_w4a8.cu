@@ -40,7 +40,9 @@ constexpr int kStages = 4;
 constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 2048;
 constexpr int kParamBytes = kTileNW4 * 12;
 constexpr int kBarrierBytes = 256;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes;
+constexpr int kFixedSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes;
+// The tile's multipliers ([K/128][128] int32) are staged in shared memory when they fit.
+constexpr int kMaxSmemGroups = (227 * 1024 - kFixedSmemBytes) / (kTileNW4 * 4);
 
 struct alignas(64) W4Params {
   CUtensorMap tmap_a[2];
@@ -53,6 +55,7 @@ struct alignas(64) W4Params {
   const float* base;      // [n_pad]
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n, n_pad;
+  int32_t mult_in_smem;  // 1: all K/128 multiplier rows of a tile fit the shared-memory table
   uint32_t* status;
 };
 
@@ -86,6 +89,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
   const uint32_t bar_tfull = bar_empty + 8 * kStages;
   const uint32_t bar_tempty = bar_tfull + 8 * kAccStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kStages + 2 * kAccStages);
+  int32_t* mult_smem = reinterpret_cast<int32_t*>(smem + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -239,6 +243,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
         param_buf[c] = v;
         thr_buf[c] = fabsf(v.y) * 0.0009765625f;
       }
+      if (p.mult_in_smem) {
+        // this tile's multipliers for every scale group: [num_kb][128] int32
+        const int4* src = reinterpret_cast<const int4*>(p.mult_t + tc.n0);
+        for (int i = et; i < num_kb * (kTileNW4 / 4); i += kEpilogueThreads) {
+          const int kb = i / (kTileNW4 / 4), c4 = i % (kTileNW4 / 4);
+          reinterpret_cast<int4*>(mult_smem)[i] = __ldg(src + static_cast<int64_t>(kb) * (p.n_pad / 4) + c4);
+        }
+      }
       asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
       const int row = tc.m0 + q * 32 + lane;
       const bool row_ok = row < p.M[tc.seg];
@@ -249,23 +261,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
       for (int j = 0; j < 64; ++j) sum[j] = 0;
       const int col0 = half * 64;
       for (int kb = 0; kb < num_kb; ++kb) {
+        const int4* mrow = p.mult_in_smem ? reinterpret_cast<const int4*>(mult_smem + kb * kTileNW4 + col0)
+                                          : reinterpret_cast<const int4*>(p.mult_t + static_cast<int64_t>(kb) * p.n_pad + tc.n0 + col0);
         w.wait(bar_tfull + 8 * acc, acc_phase);
         __syncwarp();
         tc_fence_after();
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kTileNW4 + col0;
-        const int4* mrow = reinterpret_cast<const int4*>(p.mult_t + static_cast<int64_t>(kb) * p.n_pad + tc.n0 + col0);
+        // two register buffers: the load of chunk ch + 1 is in flight while chunk ch is accumulated
+        uint32_t r[2][16];
+        tmem_ld_32x16(t_row, r[0]);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-          uint32_t r[16];
-          tmem_ld_32x16(t_row + ch * 16, r);
           tmem_wait_ld();
+          if (ch < 3) tmem_ld_32x16(t_row + (ch + 1) * 16, r[(ch + 1) & 1]);
 #pragma unroll
           for (int j4 = 0; j4 < 4; ++j4) {
-            const int4 m = __ldg(mrow + ch * 4 + j4);
+            const int4 m = mrow[ch * 4 + j4];
             const int mv[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              sum[ch * 16 + j4 * 4 + e] += static_cast<long long>(static_cast<int32_t>(r[j4 * 4 + e])) * static_cast<long long>(mv[e]);
+              sum[ch * 16 + j4 * 4 + e] +=
+                  static_cast<long long>(static_cast<int32_t>(r[ch & 1][j4 * 4 + e])) * static_cast<long long>(mv[e]);
           }
         }
         tc_fence_before();
@@ -387,14 +403,19 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
   p.n_pad = p.tiles_n * kTileNW4;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
+  const int groups = w->K / kTileK;
+  p.mult_in_smem = groups <= kMaxSmemGroups ? 1 : 0;
+  const int smem_bytes = kFixedSmemBytes + (p.mult_in_smem ? groups * kTileNW4 * 4 : 0);
   const int64_t total = tiles_m * p.tiles_n;
   const int grid = static_cast<int>(total < sms ? total : sms);
   static bool configured[16] = {};
   if (dev >= 0 && dev < 16 && !configured[dev]) {
-    if (cudaFuncSetAttribute(gemm_w4a8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return TRDQ_ERR_CUDA;
+    if (cudaFuncSetAttribute(gemm_w4a8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kFixedSmemBytes + kMaxSmemGroups * kTileNW4 * 4) != cudaSuccess)
+      return TRDQ_ERR_CUDA;
     configured[dev] = true;
   }
-  gemm_w4a8_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);
+  gemm_w4a8_kernel<<<grid, kThreads, smem_bytes, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 

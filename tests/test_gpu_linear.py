@@ -187,6 +187,7 @@ def test_linear_strided_output_and_cfg_segments():
     (129, 1168, 4608, True),     # 36 groups: accumulators rotate many times; N is not a multiple of the tile
     (1, 16, 128, False),         # one group, smallest problem
     (260, 3456, 1152, False),
+    (40, 128, 12416, True),      # 97 groups: the multiplier table no longer fits shared memory
 ])
 def test_linear_w4a8_matches_oracle(M, N, K, with_bias):
     """int4 weights with one scale per (channel, 128 k): per-group integer sums, scaled and added."""
