@@ -301,7 +301,7 @@ def run_reference(args, wl: WL.Workload):
 def run_ours(args, wl: WL.Workload):
     import torch
     import torch.distributed as dist
-    from paper_2503_06564_b200 import build as lib_build, trdq
+    from paper_2503_06564_b200 import build as lib_build, multirank, trdq
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -333,10 +333,8 @@ def run_ours(args, wl: WL.Workload):
     if world > 1:
         dist.barrier()
     ms = time_region(step, args.steps)
+    ms = multirank.max_over_ranks(ms, device="cuda")
     if world > 1:
-        tmax = torch.tensor([ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
         dist.barrier()
     # per-kernel passes (same buffers, launches back to back from a CUDA graph)
     reps = max(3, min(args.steps, 20))
@@ -367,10 +365,7 @@ def run_ours(args, wl: WL.Workload):
 
     e2e_step(0)
     ms_e2e = time_region(e2e_step, e2e_steps) / e2e_steps
-    if world > 1:
-        tmax = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_e2e = float(tmax.item())
+    ms_e2e = multirank.max_over_ranks(ms_e2e, device="cuda")
 
     peaks = load_peaks()
     in_long_step = True
