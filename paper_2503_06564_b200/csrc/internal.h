@@ -51,6 +51,11 @@ uint32_t* device_status_word();  // device address of the status word of the cur
 cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
                                    void* codes, float* scales, cudaStream_t stream);
 
+// rotate_quantize_tma.cu: per-row int8 path for rows of at most 36 blocks (TMA-staged, one thread per block)
+int rotate_quantize_tma_rows(int32_t K);  // rows per tile, 0 if K is too wide for this kernel
+trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
+                                       float* scales, cudaStream_t stream);
+
 // gemm_i8.cu
 struct GemmSegment {
   const int8_t* codes;  // dev [M,K]

@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--no-graph", action="store_true", help="time individual launches issued from Python (profiler runs)")
     args = ap.parse_args()
     build.build()
     torch.manual_seed(0)
@@ -57,13 +58,30 @@ def main():
     for i in range(args.warmup):
         run(i)
     torch.cuda.synchronize()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.iters + 1)]
-    ev[0].record()
-    for i in range(args.iters):
-        run(i)
-        ev[i + 1].record()
-    torch.cuda.synchronize()
-    ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.iters))
+    if args.no_graph:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.iters + 1)]
+        ev[0].record()
+        for i in range(args.iters):
+            run(i)
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.iters))
+    else:
+        # one pass over all buffer sets captured in a CUDA graph: launches are back to back on the
+        # device, so small shapes are not limited by the host's launch rate
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(args.sets):
+                run(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.iters + 1)]
+        ev[0].record()
+        for i in range(args.iters):
+            graph.replay()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        ms = sorted(ev[i].elapsed_time(ev[i + 1]) / args.sets for i in range(args.iters))
     med = ms[len(ms) // 2]
     assert trdq.trdq_device_status() == 0
     print(json.dumps({"kernel": args.kernel, "M": M, "K": K, "N": N if args.kernel == "gemm" else None, "wbits": args.wbits,

@@ -35,6 +35,9 @@ def _x(M, K, seed, outliers=True):
     (5, 128, 2, True),
     (33, 384, 2, True),         # 3 blocks: lane groups do not fill a warp multiple
     (3, 17408, 1, True),        # 136 blocks: several blocks per lane group
+    (100, 640, 2, True),        # 5 blocks: 56 rows per tile, the last warp is partly idle, ragged last tile
+    (9, 4736, 1, True),         # 37 blocks: too wide for one thread per block, lane-group kernel
+    (600, 1152, 1, False),      # several tiles per CTA slot: the two-stage ring wraps
 ])
 def test_rotate_quantize_matches_oracle(M, K, G, smooth):
     from paper_2503_06564_b200 import trdq
