@@ -74,6 +74,20 @@ trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_byt
   return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
+trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint32_t box_cols, uint64_t rows,
+                              uint64_t row_stride_bytes, uint32_t boxes, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return TRDQ_ERR_CUDA;
+  const CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16;
+  const cuuint64_t dims[3] = {box_cols, rows, boxes};
+  const cuuint64_t strides[2] = {row_stride_bytes, static_cast<cuuint64_t>(box_cols) * elem_bytes};
+  const cuuint32_t box[3] = {box_cols, box_rows, boxes};
+  const cuuint32_t elem_strides[3] = {1, 1, 1};
+  const CUresult r = fn(out, dt, 3, const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int find_group(const std::vector<int32_t>& bounds, int32_t t) {

@@ -80,4 +80,10 @@ trdq_status encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t ro
 trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint64_t cols, uint64_t rows,
                            uint64_t row_stride_bytes, uint32_t box_cols, uint32_t box_rows, uint32_t swizzle_bytes);
 
+// A row-major [rows, boxes * box_cols] matrix viewed as (column in box, row, box): one copy of
+// box_cols x box_rows x boxes moves a tile of box_rows full rows and stores it box after box, each box
+// being box_rows rows of box_cols elements (128 bytes), 128-byte swizzle.
+trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint32_t box_cols, uint64_t rows,
+                              uint64_t row_stride_bytes, uint32_t boxes, uint32_t box_rows);
+
 }  // namespace trdq

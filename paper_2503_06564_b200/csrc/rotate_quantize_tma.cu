@@ -26,8 +26,10 @@ constexpr int kMaxComputeThreads = 288;
 constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23
 
 struct alignas(64) RqParams {
-  CUtensorMap tmap_x;      // bf16 [M, K] (row stride ldx), box 64 x R, 128-byte swizzle
-  CUtensorMap tmap_codes;  // int8 [M, K], box 128 x R, 128-byte swizzle
+  // Both maps view a row as K/64 (K/128) column boxes: dims (column in box, row, box), so that ONE copy
+  // moves a whole R-row tile and lays it out box after box, each box R rows of 128 bytes, 128-byte swizzle.
+  CUtensorMap tmap_x;      // bf16: (64, M, K/64), box 64 x R x K/64
+  CUtensorMap tmap_codes;  // int8: (128, M, K/128), box 128 x R x K/128
   const float* vec;        // fused vector of the group, K floats
   float* scales;           // [M]
   int32_t M, K, R;         // R rows per tile, a multiple of 8
@@ -48,7 +50,10 @@ __device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
   return __byte_perm(lo, hi, 0x5410);
 }
 
-__global__ void __launch_bounds__(kMaxComputeThreads + 32, 1) rotate_quantize_tma_kernel(const __grid_constant__ RqParams p) {
+// MAXT compute threads per CTA, MINB CTAs per SM: narrow rows run two smaller CTAs per SM so that one
+// transforms while the other waits at its row-max barrier or moves data.
+template <int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT + 32, MINB) rotate_quantize_tma_kernel(const __grid_constant__ RqParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -92,7 +97,7 @@ __global__ void __launch_bounds__(kMaxComputeThreads + 32, 1) rotate_quantize_tm
         w.wait(bar_empty + 8 * stage, phase ^ 1);
         mbar_arrive_expect_tx(bar_full + 8 * stage, stage_bytes);
         const uint32_t dst = smem_base + stage * stage_bytes;
-        for (int bx = 0; bx < 2 * nb; ++bx) tma_load_2d(dst + bx * box_in_bytes, &p.tmap_x, bx * 64, tile * R, bar_full + 8 * stage);
+        tma_load_3d(dst, &p.tmap_x, 0, tile * R, 0, bar_full + 8 * stage);  // all 2 * nb column boxes in one copy
         if (++stage == 2) {
           stage = 0;
           phase ^= 1;
@@ -194,7 +199,7 @@ __global__ void __launch_bounds__(kMaxComputeThreads + 32, 1) rotate_quantize_tm
     fence_proxy_async_smem();
     asm volatile("bar.sync 2, %0;" ::"r"(p.compute_threads) : "memory");
     if (tid == 0) {
-      for (int bb = 0; bb < nb; ++bb) tma_store_2d(&p.tmap_codes, bb * TRDQ_BLOCK, tile * R, out_base + bb * box_in_bytes);  // rows >= M are clipped
+      tma_store_3d(&p.tmap_codes, 0, tile * R, 0, out_base);  // all nb column boxes; rows >= M are clipped
       bulk_commit_group();
     }
   }
@@ -204,10 +209,13 @@ __global__ void __launch_bounds__(kMaxComputeThreads + 32, 1) rotate_quantize_tm
 
 }  // namespace
 
+constexpr int kSmallComputeThreads = 144;
+
 // Rows per tile for this kernel, or 0 if the row is too wide for it.
 int rotate_quantize_tma_rows(int32_t K) {
   const int nb = K / TRDQ_BLOCK;
-  int rows = (kMaxComputeThreads / nb) / 8 * 8;
+  const int budget = kMaxComputeThreads;
+  int rows = (budget / nb) / 8 * 8;
   if (rows > 256) rows = 256;  // TMA box limit
   return rows >= 8 ? rows : 0;
 }
@@ -221,11 +229,11 @@ trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t 
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   RqParams p;
-  trdq_status st = encode_tmap_2d(&p.tmap_x, x_bf16, 2, static_cast<uint64_t>(K), static_cast<uint64_t>(M), static_cast<uint64_t>(ldx) * 2,
-                                  64, static_cast<uint32_t>(R), 128);
+  trdq_status st = encode_tmap_boxes(&p.tmap_x, x_bf16, 2, 64, static_cast<uint64_t>(M), static_cast<uint64_t>(ldx) * 2,
+                                     static_cast<uint32_t>(2 * nb), static_cast<uint32_t>(R));
   if (st != TRDQ_OK) return st;
-  st = encode_tmap_2d(&p.tmap_codes, codes, 1, static_cast<uint64_t>(K), static_cast<uint64_t>(M), static_cast<uint64_t>(K), 128,
-                      static_cast<uint32_t>(R), 128);
+  st = encode_tmap_boxes(&p.tmap_codes, codes, 1, 128, static_cast<uint64_t>(M), static_cast<uint64_t>(K), static_cast<uint32_t>(nb),
+                         static_cast<uint32_t>(R));
   if (st != TRDQ_OK) return st;
   p.vec = vec;
   p.scales = scales;
@@ -240,14 +248,22 @@ trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t 
                       3 * static_cast<size_t>(R) * 4 + 64;
   static bool configured[16] = {};
   if (dev >= 0 && dev < 16 && !configured[dev]) {
-    if (cudaFuncSetAttribute(rotate_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(rotate_quantize_tma_kernel<kMaxComputeThreads, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(rotate_quantize_tma_kernel<kSmallComputeThreads, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             113 * 1024) != cudaSuccess)
       return TRDQ_ERR_CUDA;
     configured[dev] = true;
   }
-  if (smem > 227 * 1024) return TRDQ_ERR_SHAPE;
+  const bool small = false;  // the two-CTA-per-SM variant measured slower on 9- and 18-block rows; kept for 8-block experiments
+  if (smem > (small ? 113u : 227u) * 1024) return TRDQ_ERR_SHAPE;
   const int num_tiles = (M + R - 1) / R;
-  const int grid = num_tiles < sms ? num_tiles : sms;
-  rotate_quantize_tma_kernel<<<grid, p.compute_threads + 32, smem, stream>>>(p);
+  const int slots = small ? 2 * sms : sms;
+  const int grid = num_tiles < slots ? num_tiles : slots;
+  if (small)
+    rotate_quantize_tma_kernel<kSmallComputeThreads, 2><<<grid, p.compute_threads + 32, smem, stream>>>(p);
+  else
+    rotate_quantize_tma_kernel<kMaxComputeThreads, 1><<<grid, p.compute_threads + 32, smem, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
