@@ -316,7 +316,7 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
   if (ldx < rot->K) return TRDQ_ERR_SHAPE;
   if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return TRDQ_ERR_ALIGN;
   const float* vec = rot->act_vec + static_cast<size_t>(g) * rot->K;
-  if (rotate_quantize_tma_rows(rot->K) > 0)
+  if (rotate_quantize_prefers_tma(M, rot->K))
     return launch_rotate_quantize_tma(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream));
   const cudaError_t e = launch_rotate_quantize(X_bf16, ldx, M, rot->K, vec, 0, codes, scales, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;

@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();
+  griddep_wait();  // codes, scales and weights may come from the kernel before; Y may still be read by it
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -317,8 +319,7 @@ cudaError_t launch_one(const GemmParams& p, int grid, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  gemm_w8a8_kernel<BN, MODE><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
-  return cudaGetLastError();
+  return launch_overlapped(gemm_w8a8_kernel<BN, MODE>, dim3(grid), dim3(kThreads), C::kSmemBytes, stream, p);
 }
 
 // Cost model for the tile width: waves of CTAs times the time of one tile (main loop grows

@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();
+  griddep_wait();  // codes, scales and weights may come from the kernel before; Y may still be read by it
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -415,8 +417,7 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
       return TRDQ_ERR_CUDA;
     configured[dev] = true;
   }
-  gemm_w4a8_kernel<<<grid, kThreads, smem_bytes, stream>>>(p);
-  return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return launch_overlapped(gemm_w4a8_kernel, dim3(grid), dim3(kThreads), smem_bytes, stream, p) == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
 }  // namespace trdq

@@ -53,6 +53,7 @@ cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, i
 
 // rotate_quantize_tma.cu: per-row int8 path for rows of at most 36 blocks (TMA-staged, one thread per block)
 int rotate_quantize_tma_rows(int32_t K);  // rows per tile, 0 if K is too wide for this kernel
+bool rotate_quantize_prefers_tma(int32_t M, int32_t K);
 trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
                                        float* scales, cudaStream_t stream);
 
@@ -85,5 +86,22 @@ trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_byt
 // being box_rows rows of box_cols elements (128 bytes), 128-byte swizzle.
 trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint32_t box_cols, uint64_t rows,
                               uint64_t row_stride_bytes, uint32_t boxes, uint32_t box_rows);
+
+// Launches `kernel` so that its prologue may overlap the tail of the previous kernel in the stream
+// (the kernel itself orders its memory accesses with griddep_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 }  // namespace trdq

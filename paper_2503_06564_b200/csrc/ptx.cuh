@@ -36,6 +36,15 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// ------------------------------------------------ programmatic dependent launch ----
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream is still running.  Everything that touches memory the earlier
+// kernel may read or write must come after griddep_wait(), which returns once that kernel has
+// completed and its writes are visible.  griddep_launch_dependents() lets the NEXT kernel in the
+// stream begin its own prologue early.  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier ----
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

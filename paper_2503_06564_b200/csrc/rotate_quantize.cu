@@ -13,6 +13,7 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace trdq {
 namespace {
@@ -228,6 +229,8 @@ rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, in
   for (int i = threadIdx.x; i < K / 4; i += blockDim.x) reinterpret_cast<float4*>(svec)[i] = __ldg(reinterpret_cast<const float4*>(vec) + i);
   if (threadIdx.x < 32) row_max[0][threadIdx.x] = 0u;
   __syncthreads();
+  griddep_launch_dependents();
+  griddep_wait();  // x may be written, and the code buffer still read, by the kernel before (the group vector is constant)
 
   const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
   const int col0 = b * TRDQ_BLOCK + lane4 * 8;  // first element of chunk 0 of this lane; chunk c is 32 further
@@ -348,9 +351,8 @@ cudaError_t launch_rows_fast(const void* x, int64_t ldx, int32_t M, int32_t K, c
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = min(num_tiles, sms * 2);
   const size_t smem = static_cast<size_t>(K) * sizeof(float);
-  rotate_quantize_rows_kernel<2><<<grid, threads, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), ldx, M, K, vec,
-                                                                  static_cast<int8_t*>(codes), scales, rows, 0.0f);
-  return cudaGetLastError();
+  return launch_overlapped(rotate_quantize_rows_kernel<2>, dim3(grid), dim3(threads), smem, stream, static_cast<const __nv_bfloat16*>(x),
+                           ldx, M, K, vec, static_cast<int8_t*>(codes), scales, rows, 0.0f);
 }
 
 template <int MODE, int P>

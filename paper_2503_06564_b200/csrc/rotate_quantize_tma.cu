@@ -84,6 +84,8 @@ __global__ void __launch_bounds__(MAXT + 32, MINB) rotate_quantize_tma_kernel(co
   for (int i = tid; i < p.K / 4; i += blockDim.x) reinterpret_cast<float4*>(svec)[i] = __ldg(reinterpret_cast<const float4*>(p.vec) + i);
   for (int i = tid; i < 3 * R; i += blockDim.x) row_max[i] = 0u;
   __syncthreads();
+  griddep_launch_dependents();
+  griddep_wait();  // X may be written, and the code buffer still read, by the kernel before (the group vector is constant)
 
   if (warp == compute_warps) {
     // ------------------------------------------------------------ TMA producer
@@ -220,6 +222,17 @@ int rotate_quantize_tma_rows(int32_t K) {
   return rows >= 8 ? rows : 0;
 }
 
+// The one-thread-per-block kernel keeps a whole tile of R rows in the registers of one CTA, so it needs
+// at least two tiles per SM to overlap one tile's arithmetic with the next one's loads; below that the
+// lane-group kernel, which spreads the same rows over twice as many smaller CTAs, finishes sooner.
+bool rotate_quantize_prefers_tma(int32_t M, int32_t K) {
+  const int R = rotate_quantize_tma_rows(K);
+  if (R == 0) return false;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return static_cast<int64_t>(M) >= 2ll * sms * R;
+}
+
 trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
                                        float* scales, cudaStream_t stream) {
   const int R = rotate_quantize_tma_rows(K);
@@ -260,11 +273,10 @@ trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t 
   const int num_tiles = (M + R - 1) / R;
   const int slots = small ? 2 * sms : sms;
   const int grid = num_tiles < slots ? num_tiles : slots;
-  if (small)
-    rotate_quantize_tma_kernel<kSmallComputeThreads, 2><<<grid, p.compute_threads + 32, smem, stream>>>(p);
-  else
-    rotate_quantize_tma_kernel<kMaxComputeThreads, 1><<<grid, p.compute_threads + 32, smem, stream>>>(p);
-  return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  const cudaError_t e =
+      small ? launch_overlapped(rotate_quantize_tma_kernel<kSmallComputeThreads, 2>, dim3(grid), dim3(p.compute_threads + 32), smem, stream, p)
+            : launch_overlapped(rotate_quantize_tma_kernel<kMaxComputeThreads, 1>, dim3(grid), dim3(p.compute_threads + 32), smem, stream, p);
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
 }  // namespace trdq
