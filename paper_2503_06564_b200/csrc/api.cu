@@ -242,6 +242,10 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
         trdq_weights_destroy(w);
         return st;
       }
+      if (wbits == 8 && encode_tmap_u8_sw128(&gw.tmap_b_half[i], gw.codes, row_bytes, N, row_bytes, box_bytes, kTileN[i] / 2) != TRDQ_OK) {
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_CUDA;
+      }
     }
     if (wbits == 4) {
       const int n_pad = (N + 127) / 128 * 128;

@@ -1,0 +1,59 @@
+// Dequantizing epilogue arithmetic shared by the 8-bit GEMM kernels (Eq. 10 on the codes, then the
+// per-token and per-channel scales of Sec. 3.1 and the bias).
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace trdq {
+
+// 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n], packed to bf16 pairs.
+// pb4: (sw, bias) of the 32 columns as 16 float4; thr4: 2^-10 * |bias| as 8 float4.
+__device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm, const float4* pb4, const float4* thr4,
+                                              uint32_t (&packed)[16]) {
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    const float4 p01 = pb4[j / 2], p23 = pb4[j / 2 + 1], th = thr4[j / 4];
+    const float swv[4] = {p01.x, p01.z, p23.x, p23.z};
+    const float bv[4] = {p01.y, p01.w, p23.y, p23.w};
+    const float tv[4] = {th.x, th.y, th.z, th.w};
+    float y[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int32_t a = static_cast<int32_t>(r[j + e]);
+      const float af = static_cast<float>(a);
+      const float s_hi = __fmul_rn(sxm, swv[e]);
+      float v = __fmaf_rn(af, s_hi, bv[e]);
+      // fp32 is accurate to 2^-23 of the product.  Only when product and bias cancel to less than
+      // 2^-10 of the bias can that exceed a bf16 rounding step of the result; then the scale product
+      // is carried as an exact two-term sum and the part of the accumulator that fp32 could not hold
+      // is added back.
+      if (fabsf(v) < tv[e]) {
+        const float s_lo = __fmaf_rn(sxm, swv[e], -s_hi);
+        v = __fmaf_rn(af, s_lo, v);
+        v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
+      }
+      y[e] = v;
+    }
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]);
+    const __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2], y[3]);
+    packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h0);
+    packed[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+  }
+}
+
+// Stages the epilogue parameters of `count` columns starting at n0: (sw, bias) and the cancellation threshold.
+__device__ __forceinline__ void stage_column_params(float2* pb, float* thr, const float* sw, const __nv_bfloat16* bias, int n0, int N,
+                                                    int count, int tid, int nthreads) {
+  for (int c = tid; c < count; c += nthreads) {
+    const int n = n0 + c;
+    float2 v = make_float2(0.0f, 0.0f);
+    if (n < N) {
+      v.x = __ldg(sw + n);
+      v.y = bias ? __bfloat162float(bias[n]) : 0.0f;
+    }
+    pb[c] = v;
+    thr[c] = fabsf(v.y) * 0.0009765625f;
+  }
+}
+
+}  // namespace trdq

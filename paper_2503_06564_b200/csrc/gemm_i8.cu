@@ -18,6 +18,9 @@
 // once for both.  Every wait is bounded (see BoundedWaiter).
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
+#include "epilogue.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -206,16 +209,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
       float2* pb = param_buf + acc * BN;                                           // (sw, bias)
       float* thr = reinterpret_cast<float*>(param_buf + 2 * BN) + acc * BN;        // 2^-10 * |bias|
       if (MODE == 0) {
-        for (int c = et; c < BN; c += kEpilogueThreads) {
-          const int n = tc.n0 + c;
-          float2 v = make_float2(0.0f, 0.0f);
-          if (n < p.N) {
-            v.x = __ldg(p.sw + n);
-            v.y = p.bias ? __bfloat162float(p.bias[n]) : 0.0f;
-          }
-          pb[c] = v;
-          thr[c] = fabsf(v.y) * 0.0009765625f;
-        }
+        stage_column_params(pb, thr, p.sw, p.bias, tc.n0, p.N, BN, et, kEpilogueThreads);
         asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
       }
       const int row = tc.m0 + q * 32 + lane;
@@ -237,35 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
           const float4* pb4 = reinterpret_cast<const float4*>(pb + c * 32);
           const float4* thr4 = reinterpret_cast<const float4*>(thr + c * 32);
           uint32_t packed[16];
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 p01 = pb4[j / 2], p23 = pb4[j / 2 + 1], th = thr4[j / 4];
-            const float swv[4] = {p01.x, p01.z, p23.x, p23.z};
-            const float bv[4] = {p01.y, p01.w, p23.y, p23.w};
-            const float tv[4] = {th.x, th.y, th.z, th.w};
-            float y[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int32_t a = static_cast<int32_t>(r[j + e]);
-              const float af = static_cast<float>(a);
-              const float s_hi = __fmul_rn(sxm, swv[e]);
-              float v = __fmaf_rn(af, s_hi, bv[e]);
-              // fp32 is accurate to 2^-23 of the product.  Only when product and bias cancel to less
-              // than 2^-10 of the bias can that exceed a bf16 rounding step of the result; then the
-              // scale product is carried as an exact two-term sum and the part of the accumulator
-              // that fp32 could not hold is added back.
-              if (fabsf(v) < tv[e]) {
-                const float s_lo = __fmaf_rn(sxm, swv[e], -s_hi);
-                v = __fmaf_rn(af, s_lo, v);
-                v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
-              }
-              y[e] = v;
-            }
-            const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]);
-            const __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2], y[3]);
-            packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h0);
-            packed[j / 2 + 1] = *reinterpret_cast<const uint32_t*>(&h1);
-          }
+          dequant_row32(r, sxm, pb4, thr4, packed);
           // staging tile: row = lane, 64 bytes per row, 16-byte chunk j stored at j ^ ((lane >> 1) & 3)
           if (lane == 0) bulk_wait_group_read<0>();  // the previous store has finished reading the tile
           __syncwarp();
@@ -344,6 +310,15 @@ int choose_tile_n(int64_t tiles_m, int N, int sms) {
 
 trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
                            cudaStream_t stream) {
+  // Large problems go to the CTA-pair kernel (two SMs per 256-row tile, a third less operand traffic per SM).
+  static const int pair_min_rows = [] {
+    const char* e = getenv("TRDQ_PAIR_MIN_M");
+    return e ? atoi(e) : 2048;
+  }();
+  if (!raw_i32 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows) {
+    const trdq_status st = launch_gemm_w8_pair(w, g, seg, bias_bf16, stream);
+    if (st != TRDQ_ERR_SHAPE) return st;
+  }
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

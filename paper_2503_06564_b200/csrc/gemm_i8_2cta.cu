@@ -1,0 +1,417 @@
+// INT8 GEMM + dequantizing epilogue, CTA-PAIR variant (tcgen05 cta_group::2).
+//
+// Two CTAs of a cluster (two SMs) compute one 256 x BN tile of Y.  Each CTA loads its own 128 rows of
+// the activation codes and HALF of the weight tile (BN/2 rows); one thread of the leader CTA issues
+// tcgen05.mma cta_group::2 (256 x BN x 32), which reads A and B from both CTAs' shared memory and
+// writes each CTA's 128 rows of the accumulator into that CTA's tensor memory.  Per multiply-add the
+// pair pulls 2/3 (BN = 256) of the operand bytes the single-CTA kernel pulls from L2, which is what
+// bounded that kernel (measured with operand loads removed: 2.7 -> 4.0 PTOPS at K = N = 4608).
+//
+// Synchronisation (all mbarriers; every wait bounded):
+//   full[s]    in the LEADER: both producers arrive with their byte counts; both CTAs' TMA copies
+//              complete on it (the copies carry .cta_group::2 so that they may signal the peer CTA)
+//   empty[s]   in each CTA: tcgen05.commit multicast to both CTAs when the MMAs reading stage s are done
+//   tfull[a]   in each CTA: tcgen05.commit multicast when accumulator a is complete
+//   tempty[a]  in the LEADER: the epilogue warps of both CTAs arrive (16 arrivals)
+// The epilogue is the single-CTA kernel's (one row per thread, eight warps per CTA), with two staging
+// tiles per warp so that a TMA store overlaps the next chunk's arithmetic.  No TMA multicast is used.
+#include <cuda_bf16.h>
+
+#include "epilogue.cuh"
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace trdq {
+namespace {
+
+constexpr int kTileM = 128;       // rows per CTA; the pair covers 256
+constexpr int kTileKBytes = 128;
+constexpr int kUmmaK = 32;
+constexpr int kThreads = 384;
+constexpr int kEpilogueThreads = 256;
+constexpr int kAccStride = 256;
+constexpr int kTmemCols = 512;
+constexpr int kSmemBudget = 227 * 1024;
+
+template <int BN>
+struct Cfg2 {
+  static constexpr int kABytes = kTileM * kTileKBytes;
+  static constexpr int kBBytes = (BN / 2) * kTileKBytes;  // this CTA's half of the weight tile
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kParamBytes = 2 * BN * 12;
+  static constexpr int kBarrierBytes = 256;
+  static constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 2 * 2048;  // two 32 x 32 bf16 tiles per warp
+  static constexpr int kStages = (kSmemBudget - 1024 - kOutStageBytes - kParamBytes - kBarrierBytes) / kStageBytes;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes;
+  static_assert(kStages >= 3 && kStages <= 10, "stage count out of range");
+  static_assert(kStageBytes % 1024 == 0, "stage tiles must stay 1024-byte aligned");
+};
+
+struct alignas(64) Gemm2Params {
+  CUtensorMap tmap_a[2];    // codes of each segment, box 128 B x 128 rows
+  CUtensorMap tmap_b;       // weights, box 128 B x BN/2 rows
+  CUtensorMap tmap_out[2];  // bf16 output, box 32 x 32, 64-byte swizzle
+  const float* sx[2];
+  int32_t M[2];
+  int32_t pair_tiles_m[2];  // 256-row tiles per segment
+  const float* sw;
+  const __nv_bfloat16* bias;
+  int32_t N, K, tiles_n;
+  uint32_t* status;
+};
+
+struct TileCoord {
+  int seg, m0, n0;
+};
+__device__ __forceinline__ TileCoord pair_tile_coord(const Gemm2Params& p, int tile, int bn) {
+  const int tiles_m = p.pair_tiles_m[0] + p.pair_tiles_m[1];
+  const int nt = tile / tiles_m;
+  int mt = tile - nt * tiles_m;
+  TileCoord c;
+  c.seg = mt >= p.pair_tiles_m[0] ? 1 : 0;
+  if (c.seg) mt -= p.pair_tiles_m[0];
+  c.m0 = mt * 2 * kTileM;
+  c.n0 = nt * bn;
+  return c;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_remote_arrive(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_remote_arrive_expect_tx(uint32_t cluster_addr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// TMA load into THIS CTA's shared memory whose completion is counted on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* tmap, int32_t x, int32_t y, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t"
+      "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in BOTH CTAs once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(static_cast<uint16_t>(3))
+               : "memory");
+}
+// kind::i8 instruction descriptor for the pair: M = 256.
+__host__ __device__ constexpr uint32_t umma_idesc_s8_pair(int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
+}
+
+template <int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8a8_pair_kernel(const __grid_constant__ Gemm2Params p) {
+  using C = Cfg2<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t out_stage_base = smem_base + C::kStages * C::kStageBytes;
+  float2* param_buf = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes + C::kOutStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes + C::kOutStageBytes + C::kParamBytes);
+  const uint32_t bar_full = smem_u32(bars);                  // [S]   used in the leader
+  const uint32_t bar_empty = bar_full + 8 * C::kStages;      // [S]   each CTA's own
+  const uint32_t bar_tfull = bar_empty + 8 * C::kStages;     // [2]   each CTA's own
+  const uint32_t bar_tempty = bar_tfull + 16;                // [2]   used in the leader
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::kStages + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
+  const int total_tiles = (p.pair_tiles_m[0] + p.pair_tiles_m[1]) * p.tiles_n;
+  const int num_kb = p.K / kTileKBytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 2);   // one arrive.expect_tx from each CTA's producer
+      mbar_init(bar_empty + 8 * s, 1);  // one multicast commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, 2 * (kEpilogueThreads / 32));  // epilogue warps of both CTAs
+    }
+    fence_mbar_init();
+  }
+  if (warp == 2) {
+    tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised and its tensor memory allocated before anything is signalled
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();
+  griddep_wait();
+
+  if (warp == 0) {
+    // ---------------------------------------------------- TMA producer (both CTAs)
+    if (elect_one()) {
+      prefetch_tensormap(&p.tmap_a[0]);
+      prefetch_tensormap(&p.tmap_a[1]);
+      prefetch_tensormap(&p.tmap_b);
+      prefetch_tensormap(&p.tmap_out[0]);
+      prefetch_tensormap(&p.tmap_out[1]);
+      BoundedWaiter w(p.status, kStatusTimeoutProducer);
+      const uint32_t leader_full = map_to_cta(bar_full, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int tile = cluster_id; tile < total_tiles; tile += num_clusters) {
+        const TileCoord tc = pair_tile_coord(p, tile, BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          w.wait(bar_empty + 8 * stage, phase ^ 1);
+          const uint32_t a_dst = smem_base + stage * C::kStageBytes;
+          const uint32_t b_dst = a_dst + C::kABytes;
+          const uint32_t full_s = leader_full + 8 * stage;
+          mbar_remote_arrive_expect_tx(full_s, C::kStageBytes);
+          tma_load_2d_pair(a_dst, &p.tmap_a[tc.seg], kb * kTileKBytes, tc.m0 + rank * kTileM, full_s);
+          tma_load_2d_pair(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0 + rank * (BN / 2), full_s);
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+      }
+      w.settle();
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------- MMA issuer (leader only)
+    if (leader && elect_one()) {
+      BoundedWaiter w(p.status, kStatusTimeoutMma);
+      constexpr uint32_t idesc = umma_idesc_s8_pair(BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (int tile = cluster_id; tile < total_tiles; tile += num_clusters) {
+        w.wait(bar_tempty + 8 * acc, acc_phase ^ 1);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kAccStride;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          w.wait(bar_full + 8 * stage, phase);
+          tc_fence_after();
+          const uint32_t a_addr = smem_base + stage * C::kStageBytes;
+          const uint64_t a_desc = umma_desc_k_sw128(a_addr);
+          const uint64_t b_desc = umma_desc_k_sw128(a_addr + C::kABytes);
+#pragma unroll
+          for (int k = 0; k < kTileKBytes / kUmmaK; ++k) umma_i8_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(bar_empty + 8 * stage);
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+        umma_commit_pair(bar_tfull + 8 * acc);
+        if (++acc == 2) {
+          acc = 0;
+          acc_phase ^= 1;
+        }
+      }
+      w.settle();
+    }
+  } else if (warp >= 4) {
+    // ---------------------------------------------------- epilogue (both CTAs, own 128 rows)
+    const int ew = warp - 4;
+    const int q = ew & 3;
+    const int half = ew >> 2;
+    const int et = threadIdx.x - 4 * 32;
+    constexpr int kChunksPerWarp = BN / 64;
+    const uint32_t my_stage = out_stage_base + ew * 4096;
+    const uint32_t leader_tempty = map_to_cta(bar_tempty, 0);
+    BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    uint32_t flip = 0;
+    for (int tile = cluster_id; tile < total_tiles; tile += num_clusters) {
+      const TileCoord tc = pair_tile_coord(p, tile, BN);
+      const int m0 = tc.m0 + rank * kTileM;
+      float2* pb = param_buf + acc * BN;
+      float* thr = reinterpret_cast<float*>(param_buf + 2 * BN) + acc * BN;
+      stage_column_params(pb, thr, p.sw, p.bias, tc.n0, p.N, BN, et, kEpilogueThreads);
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+      const int row = m0 + q * 32 + lane;
+      const float sxm = row < p.M[tc.seg] ? __ldg(p.sx[tc.seg] + row) : 0.0f;
+
+      w.wait(bar_tfull + 8 * acc, acc_phase);
+      __syncwarp();
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccStride;
+#pragma unroll 1
+      for (int cc = 0; cc < kChunksPerWarp; ++cc) {
+        const int c = half * kChunksPerWarp + cc;
+        uint32_t r[32];
+        tmem_ld_32x32(t_row + c * 32, r);
+        tmem_wait_ld();
+        uint32_t packed[16];
+        dequant_row32(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed);
+        const uint32_t tile_smem = my_stage + flip * 2048;
+        flip ^= 1;
+        if (lane == 0) bulk_wait_group_read<1>();  // the store issued two chunks ago has finished reading this tile
+        __syncwarp();
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          st_shared_v4(tile_smem + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4), packed[4 * v], packed[4 * v + 1], packed[4 * v + 2],
+                       packed[4 * v + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&p.tmap_out[tc.seg], tc.n0 + c * 32, m0 + q * 32, tile_smem);  // rows >= M and columns >= N are clipped
+          bulk_commit_group();
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_remote_arrive(leader_tempty + 8 * acc);
+      if (++acc == 2) {
+        acc = 0;
+        acc_phase ^= 1;
+      }
+    }
+    if (lane == 0) bulk_wait_group<0>();
+    w.settle();
+  }
+
+  // Neither CTA may release its shared or tensor memory while the other's MMAs or copies can still touch it.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
+template <int BN>
+cudaError_t launch_pair(const Gemm2Params& p, int clusters, cudaStream_t stream) {
+  using C = Cfg2<BN>;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * clusters);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_w8a8_pair_kernel<BN>, p);
+}
+
+// Clusters of two CTAs that can be resident at once (at most SMs / 2; fewer if a GPC has an odd SM count).
+template <int BN>
+int max_clusters(int dev) {
+  static int cached[16] = {};
+  if (dev < 0 || dev >= 16) return 0;
+  if (cached[dev] == 0) {
+    using C = Cfg2<BN>;
+    if (cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) {
+      cudaGetLastError();
+      cached[dev] = -1;
+      return 0;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_w8a8_pair_kernel<BN>, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      cached[dev] = -1;
+      return 0;
+    }
+    cached[dev] = n;
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+}  // namespace
+
+// Returns TRDQ_ERR_SHAPE when the pair kernel does not apply (caller falls back to the single-CTA kernel).
+trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
+  Gemm2Params p;
+  int64_t tiles_m = 0;
+  for (int s = 0; s < 2; ++s) {
+    p.sx[s] = seg[s].sx;
+    p.M[s] = seg[s].M;
+    p.pair_tiles_m[s] = (seg[s].M + 2 * kTileM - 1) / (2 * kTileM);
+    tiles_m += p.pair_tiles_m[s];
+  }
+  if (tiles_m == 0) return TRDQ_OK;
+  // tile width by the same wave model as the single-CTA kernel, over the resident clusters
+  int best = -1;
+  double best_cost = 1e300;
+  int clusters_of[kNumTileN];
+  for (int i = 0; i < kNumTileN; ++i) {
+    const int bn = kTileN[i];
+    clusters_of[i] = bn == 128 ? max_clusters<128>(dev) : bn == 192 ? max_clusters<192>(dev) : max_clusters<256>(dev);
+    if (clusters_of[i] <= 0) continue;
+    const int64_t tiles = tiles_m * ((w->N + bn - 1) / bn);
+    const int64_t waves = (tiles + clusters_of[i] - 1) / clusters_of[i];
+    const double cost = static_cast<double>(waves) * (bn + 24.0);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = i;
+    }
+  }
+  if (best < 0) return TRDQ_ERR_SHAPE;
+  const int bn = kTileN[best];
+  for (int s = 0; s < 2; ++s) {
+    const GemmSegment& src = seg[s].M > 0 ? seg[s] : seg[1 - s];
+    trdq_status st = encode_tmap_u8_sw128(&p.tmap_a[s], src.codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(src.M),
+                                          static_cast<uint64_t>(w->K), kTileKBytes, kTileM);
+    if (st != TRDQ_OK) return st;
+    st = encode_tmap_2d(&p.tmap_out[s], src.out, 2, static_cast<uint64_t>(w->N), static_cast<uint64_t>(src.M),
+                        static_cast<uint64_t>(src.ld) * 2, 32, 32, 64);
+    if (st != TRDQ_OK) return st;
+  }
+  p.tmap_b = w->groups[g].tmap_b_half[best];
+  p.sw = w->groups[g].scales;
+  p.bias = static_cast<const __nv_bfloat16*>(bias_bf16);
+  p.N = w->N;
+  p.K = w->K;
+  p.tiles_n = (w->N + bn - 1) / bn;
+  p.status = device_status_word();
+  if (!p.status) return TRDQ_ERR_CUDA;
+  const int64_t total = tiles_m * p.tiles_n;
+  const int clusters = static_cast<int>(total < clusters_of[best] ? total : clusters_of[best]);
+  const cudaError_t e = bn == 128 ? launch_pair<128>(p, clusters, stream) : bn == 192 ? launch_pair<192>(p, clusters, stream) : launch_pair<256>(p, clusters, stream);
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+}  // namespace trdq

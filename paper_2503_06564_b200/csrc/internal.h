@@ -27,6 +27,7 @@ struct GroupWeights {
   void* codes = nullptr;                // dev int8 [N,K] or packed uint8 [N,K/2]
   float* scales = nullptr;              // dev fp32 [N] or [N,K/128]
   CUtensorMap tmap_b[kNumTileN];        // TMA descriptors of `codes`, one per tile width (4-bit: only [0], 128 rows x 64 bytes)
+  CUtensorMap tmap_b_half[kNumTileN];   // 8-bit only: boxes of half a tile width (64 / 96 / 128 rows) for the CTA-pair kernel
   // 4-bit weights only: the scales of an output channel as integers on a common power-of-two grid,
   //   scales[n][kg] = mult_t[kg][n] * base[n]   (exact whenever the exponents of a channel span < 7 bits)
   int32_t* mult_t = nullptr;            // dev int32 [K/128][n_pad], n_pad = N rounded up to 128
@@ -69,6 +70,9 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
                            cudaStream_t stream);
 trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
                            cudaStream_t stream);
+// gemm_i8_2cta.cu: CTA-pair kernel; TRDQ_ERR_SHAPE means "not applicable here, use the single-CTA kernel"
+trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
+                                cudaStream_t stream);
 cudaError_t launch_w4_multipliers(const float* scales, int32_t N, int32_t groups, int32_t n_pad, int32_t* mult_t, float* base,
                                   cudaStream_t stream);
 

@@ -99,6 +99,8 @@ def test_int32_accumulators_extreme_codes():
     (200, 1152, 4608, True),
     (1, 16, 128, True),
     (77, 1040, 256, True),
+    (2304, 1152, 1152, True),    # enough rows for the CTA-pair kernel: nine 256-row tiles
+    (2100, 1040, 256, False),    # pair kernel, ragged: the last pair's second CTA has no valid row; N not a tile multiple
 ])
 def test_linear_matches_oracle(M, N, K, with_bias):
     import torch
@@ -172,6 +174,18 @@ def test_linear_strided_output_and_cfg_segments():
     assert empty[0].shape[0] == 0 and torch.equal(empty[1], y)
     # M == 0
     assert trdq.trdq_linear(wts, t, codes[:0], scales[:0], bias_d).shape == (0, N)
+    # the same through the CTA-pair kernel (>= 2048 rows in total): two segments of 1300 and 1100 rows
+    xl = _acts(2400, K, 8)
+    cl, sl = trdq.trdq_rotate_quantize(rot, t, to_dev_bf16(xl))
+    yl = trdq.trdq_linear(wts, t, cl, sl, bias_d)
+    hl = trdq.trdq_linear_cfg(wts, t, [cl[:1300].contiguous(), cl[1300:].contiguous()], [sl[:1300].contiguous(), sl[1300:].contiguous()],
+                              bias_d)
+    assert torch.equal(torch.cat(hl), yl)
+    act_l, qw_l, sw_l = ref[1]
+    rows = np.concatenate([np.arange(0, 300), np.arange(1200, 1400), np.arange(2300, 2400)])
+    q_l, sx_l = O.rotate_quantize(xl, act_l)
+    y_l_ref = O.linear_w8_rows(q_l, sx_l, qw_l, sw_l, bias, rows)
+    check_output(bf16_to_f32_np(yl)[rows], y_l_ref, max_ulp=1.0)
     # errors
     with pytest.raises(trdq.TrdqError) as e:
         trdq.trdq_linear(wts, 5000, codes, scales, bias_d)
