@@ -249,3 +249,18 @@ def test_linear_w4a8_group_scales_of_very_different_size():
     y = trdq.trdq_linear(wts, 0, codes, scales, None)
     y_ref = O.linear_w4_rows(q_ref, sx_ref, packed_ref, sw4_ref, None, np.arange(M))
     check_output(bf16_to_f32_np(y), y_ref, max_ulp=1.0)
+
+
+def test_small_shapes_through_the_cta_pair_kernel():
+    """The CTA-pair kernel normally serves problems of >= 2048 rows.  Re-run this file's 8-bit cases in a
+    child process with the threshold lowered to one row (the library reads TRDQ_PAIR_MIN_M once), so that
+    every small and ragged shape above also goes through the pair kernel."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, TRDQ_PAIR_MIN_M="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-m", "gpu", "-x", "-q", "-k",
+                          "not w4a8 and not through_the_cta_pair", "--timeout", "300"], cwd=root, env=env,
+                         capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
