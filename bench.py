@@ -371,6 +371,8 @@ def run_ours(args, wl: WL.Workload):
     in_long_step = True
     bf16_peak = peaks["bf16_tflops_sustained"] if in_long_step else peaks["bf16_tflops"]
     int8_peak = bf16_peak * INT8_OVER_BF16
+    gemm_kernel = "gemm_w4a8_kernel" if wl.wbits == 4 else ("gemm_w8a8_pair_kernel" if wl.M >= 2048 else "gemm_w8a8_kernel")
+    rq_kernel = "rotate_quantize_tma_kernel" if wl.M >= 9472 else "rotate_quantize_rows_kernel"
     gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
     rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
     line = {
@@ -384,10 +386,10 @@ def run_ours(args, wl: WL.Workload):
         "rotate_quantize_gbs": rq_gbs,
         "gemm_tops": gemm_tops,
         "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
-        "roofline": {"kernel": "gemm_w8a8_kernel", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
+        "roofline": {"kernel": gemm_kernel, "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
                      "unit": "TOPS", "frac": gemm_tops / int8_peak, "traffic": None,
                      "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
-        "roofline_rotate_quantize": {"kernel": "rotate_quantize_kernel", "bound": "hbm", "achieved": rq_gbs,
+        "roofline_rotate_quantize": {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
                                      "traffic": None, "peak_source": peaks["_source"]},
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,

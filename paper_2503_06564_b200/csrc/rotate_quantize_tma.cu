@@ -268,7 +268,7 @@ trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t 
       return TRDQ_ERR_CUDA;
     configured[dev] = true;
   }
-  const bool small = false;  // the two-CTA-per-SM variant measured slower on 9- and 18-block rows; kept for 8-block experiments
+  const bool small = false;  // two smaller CTAs per SM measured slower on 9- and 18-block rows, as did twelve compute warps with a one-stage ring
   if (smem > (small ? 113u : 227u) * 1024) return TRDQ_ERR_SHAPE;
   const int num_tiles = (M + R - 1) / R;
   const int slots = small ? 2 * sms : sms;
