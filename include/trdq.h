@@ -143,6 +143,22 @@ trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* cons
                             const int32_t M[2], const void* bias_bf16, void* const Y_bf16[2], const int64_t ldy[2],
                             void* stream);
 
+/* Split-K form of trdq_linear for problems with few rows and a long reduction (for example the
+ * cross-attention K / V projections of 960 text rows with K = 4096, which give only 72 output tiles
+ * for 148 SMs): the k range of Eq. 10's integer sum is cut into `splits` parts computed by different
+ * CTAs, their exact int32 partial sums go to a caller-provided workspace, and a second kernel adds
+ * them and applies the epilogue.  Integer addition is associative, so the output is bit-identical to
+ * trdq_linear's.  8-bit weights, one row segment.
+ * trdq_linear_splitk_workspace reports how many parts the library would use for M rows (1 = split-K does
+ * not pay for this shape) and the workspace bytes needed (splits * M * N * 4; 0 when splits == 1).
+ * trdq_linear_splitk: workspace is dev memory, 16-byte aligned, of at least that many bytes
+ * (TRDQ_ERR_NOMEM if smaller); with splits == 1 it is not touched and the call is trdq_linear.
+ * The workspace is written and read on `stream`; concurrent calls must not share it. */
+trdq_status trdq_linear_splitk_workspace(const trdq_weights* w, int32_t M, int32_t* splits, uint64_t* bytes);
+trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
+                               const void* bias_bf16, void* Y_bf16, int64_t ldy, void* workspace, uint64_t workspace_bytes,
+                               void* stream);
+
 /* One quantized linear layer of a denoising step: rotate + quantize X into the caller's code and
  * scale buffers, then the integer GEMM with its epilogue into Y (shapes as in the two calls above). */
 typedef struct trdq_layer_op {

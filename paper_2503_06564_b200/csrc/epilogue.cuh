@@ -6,6 +6,22 @@
 
 namespace trdq {
 
+// One output: y = acc * sx * sw + bias in fp32.  fp32 is accurate to 2^-23 of the product; only when
+// product and bias cancel below `thr` = 2^-10 |bias| can that exceed a bf16 rounding step of the result;
+// then the scale product is carried as an exact two-term sum and the part of the accumulator that
+// fp32 could not hold is added back.
+__device__ __forceinline__ float dequant_one(int32_t a, float sxm, float swn, float biasn, float thr) {
+  const float af = static_cast<float>(a);
+  const float s_hi = __fmul_rn(sxm, swn);
+  float v = __fmaf_rn(af, s_hi, biasn);
+  if (fabsf(v) < thr) {
+    const float s_lo = __fmaf_rn(sxm, swn, -s_hi);
+    v = __fmaf_rn(af, s_lo, v);
+    v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
+  }
+  return v;
+}
+
 // 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n], packed to bf16 pairs.
 // pb4: (sw, bias) of the 32 columns as 16 float4; thr4: 2^-10 * |bias| as 8 float4.
 __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm, const float4* pb4, const float4* thr4,
@@ -18,22 +34,7 @@ __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm
     const float tv[4] = {th.x, th.y, th.z, th.w};
     float y[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int32_t a = static_cast<int32_t>(r[j + e]);
-      const float af = static_cast<float>(a);
-      const float s_hi = __fmul_rn(sxm, swv[e]);
-      float v = __fmaf_rn(af, s_hi, bv[e]);
-      // fp32 is accurate to 2^-23 of the product.  Only when product and bias cancel to less than
-      // 2^-10 of the bias can that exceed a bf16 rounding step of the result; then the scale product
-      // is carried as an exact two-term sum and the part of the accumulator that fp32 could not hold
-      // is added back.
-      if (fabsf(v) < tv[e]) {
-        const float s_lo = __fmaf_rn(sxm, swv[e], -s_hi);
-        v = __fmaf_rn(af, s_lo, v);
-        v = __fmaf_rn(static_cast<float>(a - __float2int_rz(af)), s_hi, v);
-      }
-      y[e] = v;
-    }
+    for (int e = 0; e < 4; ++e) y[e] = dequant_one(static_cast<int32_t>(r[j + e]), sxm, swv[e], bv[e], tv[e]);
     const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]);
     const __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2], y[3]);
     packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h0);

@@ -65,17 +65,24 @@ struct alignas(64) GemmParams {
   const float* sw;
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n;
+  // split-K (raw-accumulator mode only): the k-blocks are cut into `splits` ranges of `kb_per_split`; split s
+  // writes its partial sums at out + s * split_stride (elements).  splits = 1 is the ordinary GEMM.
+  int32_t splits, kb_per_split;
+  int64_t split_stride;
   uint32_t* status;
 };
 
 struct TileCoord {
-  int seg, m0, n0;
+  int seg, m0, n0, split;
 };
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, int bn) {
   const int tiles_m = p.tiles_m[0] + p.tiles_m[1];
+  const int per_split = tiles_m * p.tiles_n;
+  TileCoord c;
+  c.split = tile / per_split;
+  tile -= c.split * per_split;
   const int nt = tile / tiles_m;
   int mt = tile - nt * tiles_m;
-  TileCoord c;
   c.seg = mt >= p.tiles_m[0] ? 1 : 0;
   if (c.seg) mt -= p.tiles_m[0];
   c.m0 = mt * kTileM;
@@ -102,8 +109,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_tiles = (p.tiles_m[0] + p.tiles_m[1]) * p.tiles_n;
-  const int num_kb = p.K / kTileKBytes;
+  const int total_tiles = (p.tiles_m[0] + p.tiles_m[1]) * p.tiles_n * p.splits;
+  const int num_kb_all = p.K / kTileKBytes;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -140,7 +147,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
       uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         const TileCoord tc = tile_coord(p, tile, BN);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const int kb0 = tc.split * p.kb_per_split;
+        const int kb1 = min(kb0 + p.kb_per_split, num_kb_all);
+        for (int kb = kb0; kb < kb1; ++kb) {
           w.wait(bar_empty + 8 * stage, phase ^ 1);
           const uint32_t a_dst = smem_base + stage * C::kStageBytes;
           const uint32_t b_dst = a_dst + C::kABytes;
@@ -168,6 +177,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
         w.wait(bar_tempty + 8 * acc, acc_phase ^ 1);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
+        const int num_kb = min(p.kb_per_split, num_kb_all - (tile / ((p.tiles_m[0] + p.tiles_m[1]) * p.tiles_n)) * p.kb_per_split);
         for (int kb = 0; kb < num_kb; ++kb) {
           w.wait(bar_full + 8 * stage, phase);
           tc_fence_after();
@@ -246,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
             bulk_commit_group();
           }
         } else if (row_ok) {
-          int32_t* out = static_cast<int32_t*>(p.out[tc.seg]) + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
+          int32_t* out = static_cast<int32_t*>(p.out[tc.seg]) + tc.split * p.split_stride + static_cast<int64_t>(row) * p.ld[tc.seg] + n_base;
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
             if (n_base + 4 * v < p.N)
@@ -356,6 +366,9 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
+  p.splits = 1;
+  p.kb_per_split = w->K / kTileKBytes;
+  p.split_stride = 0;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   const int64_t total = tiles_m * p.tiles_n;
@@ -367,6 +380,110 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
   } else {
     e = bn == 128 ? launch_one<128, 0>(p, grid, stream) : bn == 192 ? launch_one<192, 0>(p, grid, stream) : launch_one<256, 0>(p, grid, stream);
   }
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K for problems with too few output tiles to fill the GPU (few rows, long K): the k-blocks
+// are divided among `splits` CTAs per output tile, each writes exact int32 partial sums to a
+// workspace, and a second kernel adds them (integer addition: the result does not depend on the
+// order) and applies the same dequantizing arithmetic as the fused epilogue.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+__global__ void __launch_bounds__(256) splitk_reduce_epilogue_kernel(const int32_t* __restrict__ part, int splits, int64_t split_stride, int M,
+                                                                     int N, const float* __restrict__ sx, const float* __restrict__ sw,
+                                                                     const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ y,
+                                                                     int64_t ldy) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int vec_per_row = N / 8;  // N is a multiple of 16
+  const int64_t total = static_cast<int64_t>(M) * vec_per_row;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int m = static_cast<int>(i / vec_per_row);
+    const int n = static_cast<int>(i - static_cast<int64_t>(m) * vec_per_row) * 8;
+    int32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int s = 0; s < splits; ++s) {
+      const int4* src = reinterpret_cast<const int4*>(part + s * split_stride + static_cast<int64_t>(m) * N + n);
+      const int4 a = src[0], b = src[1];
+      acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+      acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+    }
+    const float sxm = __ldg(sx + m);
+    uint32_t packed[4];
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      float v2[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const float swn = __ldg(sw + n + e + u);
+        const float bn = bias ? __bfloat162float(bias[n + e + u]) : 0.0f;
+        v2[u] = dequant_one(acc[e + u], sxm, swn, bn, fabsf(bn) * 0.0009765625f);
+      }
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v2[0], v2[1]);
+      packed[e / 2] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(y + static_cast<int64_t>(m) * ldy + n) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+  }
+}
+
+}  // namespace
+
+// Number of k-ranges worth using for an M-row problem on the current device (1 = split-K does not pay).
+int splitk_choose(const trdq_weights* w, int32_t M) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t tiles = static_cast<int64_t>((M + kTileM - 1) / kTileM) * ((w->N + 127) / 128);
+  const int num_kb = w->K / kTileKBytes;
+  if (w->wbits != 8 || tiles <= 0 || tiles * 2 > sms) return 1;
+  int splits = static_cast<int>(sms / tiles);
+  if (splits > 8) splits = 8;
+  while (splits > 1 && num_kb / splits < 4) --splits;  // at least four k-blocks per range
+  if (splits < 1) splits = 1;
+  const int per = (num_kb + splits - 1) / splits;
+  return (num_kb + per - 1) / per;  // no empty range
+}
+
+trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,
+                                  int32_t* workspace, cudaStream_t stream) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  GemmParams p;
+  p.sx[0] = p.sx[1] = nullptr;
+  p.out[0] = p.out[1] = workspace;
+  p.ld[0] = p.ld[1] = w->N;
+  p.M[0] = seg.M;
+  p.M[1] = 0;
+  p.tiles_m[0] = (seg.M + kTileM - 1) / kTileM;
+  p.tiles_m[1] = 0;
+  trdq_status st = encode_tmap_u8_sw128(&p.tmap_a[0], seg.codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(seg.M),
+                                        static_cast<uint64_t>(w->K), kTileKBytes, kTileM);
+  if (st != TRDQ_OK) return st;
+  p.tmap_a[1] = p.tmap_a[0];
+  p.tmap_out[0] = p.tmap_out[1] = p.tmap_a[0];  // unused in the raw-accumulator mode
+  p.tmap_b = w->groups[g].tmap_b[0];             // 128-column tiles
+  p.sw = nullptr;
+  p.bias = nullptr;
+  p.N = w->N;
+  p.K = w->K;
+  p.tiles_n = (w->N + 127) / 128;
+  const int num_kb = w->K / kTileKBytes;
+  p.kb_per_split = (num_kb + splits - 1) / splits;
+  p.splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;
+  p.split_stride = static_cast<int64_t>(seg.M) * w->N;
+  p.status = device_status_word();
+  if (!p.status) return TRDQ_ERR_CUDA;
+  const int64_t total = static_cast<int64_t>(p.tiles_m[0]) * p.tiles_n * p.splits;
+  const int grid = static_cast<int>(total < sms ? total : sms);
+  if (launch_one<128, 1>(p, grid, stream) != cudaSuccess) return TRDQ_ERR_CUDA;
+  const int64_t vecs = static_cast<int64_t>(seg.M) * (w->N / 8);
+  int64_t rgrid = (vecs + 255) / 256;
+  if (rgrid > static_cast<int64_t>(sms) * 8) rgrid = static_cast<int64_t>(sms) * 8;
+  const cudaError_t e = launch_overlapped(splitk_reduce_epilogue_kernel, dim3(static_cast<unsigned>(rgrid)), dim3(256), 0, stream,
+                                          static_cast<const int32_t*>(workspace), p.splits, p.split_stride, seg.M, w->N, seg.sx,
+                                          static_cast<const float*>(w->groups[g].scales), static_cast<const __nv_bfloat16*>(bias_bf16),
+                                          static_cast<__nv_bfloat16*>(seg.out), seg.ld);
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 

@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--splitk", action="store_true", help="gemm: use trdq_linear_splitk with a preallocated workspace")
     ap.add_argument("--no-graph", action="store_true", help="time individual launches issued from Python (profiler runs)")
     args = ap.parse_args()
     build.build()
@@ -51,9 +52,15 @@ def main():
         for s in range(args.sets):
             trdq.trdq_rotate_quantize(rot, 0, xs[s], codes[s], scales[s])
 
+        splits, nbytes = trdq.trdq_linear_splitk_workspace(wts, M)
+        ws = torch.empty((max(nbytes, 16),), dtype=torch.uint8, device="cuda")
+
         def run(i):
             s = i % args.sets
-            trdq.trdq_linear(wts, 0, codes[s], scales[s], bias, ys[s])
+            if args.splitk:
+                trdq.trdq_linear_splitk(wts, 0, codes[s], scales[s], bias, ys[s], ws)
+            else:
+                trdq.trdq_linear(wts, 0, codes[s], scales[s], bias, ys[s])
         work, unit = 2.0 * M * N * K / 1e12, "TOPS"
     for i in range(args.warmup):
         run(i)

@@ -27,7 +27,7 @@ EXPORTS = (
     "trdq_find_group", "trdq_prepare_weights", "trdq_weights_destroy", "trdq_weights_info", "trdq_weights_view",
     "trdq_weights_export",
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
-    "trdq_run_layers",
+    "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk",
 )
 
 
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
                                       C.POINTER(i64), vp]
         l.trdq_gemm_i32.argtypes = [vp, i32, vp, i32, vp, i64, vp]
         l.trdq_run_layers.argtypes = [C.POINTER(LayerOp), i32, i32, vp]
+        l.trdq_linear_splitk_workspace.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_uint64)]
+        l.trdq_linear_splitk.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp, C.c_uint64, vp]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -227,6 +229,30 @@ def trdq_linear_cfg(w: Weights, t: int, codes2, scales2, bias_bf16=None, out2=No
                                  i64_2(*[int(o.stride(0)) if m > 1 else w.N for o, m in zip(out2, Ms)]), _stream()),
            "trdq_linear_cfg")
     return out2
+
+
+def trdq_linear_splitk_workspace(w: Weights, M: int) -> Tuple[int, int]:
+    """(number of k ranges, workspace bytes) the split-K call would use for M rows."""
+    splits, nbytes = C.c_int32(0), C.c_uint64(0)
+    _check(lib().trdq_linear_splitk_workspace(w._h, int(M), C.byref(splits), C.byref(nbytes)), "trdq_linear_splitk_workspace")
+    return splits.value, nbytes.value
+
+
+def trdq_linear_splitk(w: Weights, t: int, codes, scales, bias_bf16=None, out=None, workspace=None):
+    """trdq_linear with the reduction split over several CTAs per tile; `workspace` is a device tensor of at least
+    the size trdq_linear_splitk_workspace reports (allocated here when omitted)."""
+    import torch
+    M = int(codes.shape[0])
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.bfloat16, device=codes.device)
+    splits, nbytes = trdq_linear_splitk_workspace(w, M)
+    if workspace is None and nbytes:
+        workspace = torch.empty((nbytes,), dtype=torch.uint8, device=codes.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    ldy = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_linear_splitk(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, _ptr(workspace),
+                                    ws_bytes, _stream()), "trdq_linear_splitk")
+    return out
 
 
 def trdq_gemm_i32(w: Weights, t: int, codes, out=None):

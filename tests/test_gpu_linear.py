@@ -264,3 +264,37 @@ def test_small_shapes_through_the_cta_pair_kernel():
                           "not w4a8 and not through_the_cta_pair", "--timeout", "300"], cwd=root, env=env,
                          capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (960, 1152, 4096),     # cross-attention K / V projection: 72 output tiles, two k ranges
+    (256, 1024, 1024),     # single-layer configuration: 16 tiles, the eight k-blocks split in two
+    (130, 272, 4608),      # ragged rows and columns, 36 k-blocks over several ranges
+    (4096, 1152, 1152),    # enough tiles: split-K declines (one range) and the call is the ordinary GEMM
+])
+def test_linear_splitk_is_bit_identical(M, N, K):
+    """Partial int32 sums from several CTAs per tile, added by a second kernel: integer addition does not
+    depend on the order, so the output must equal trdq_linear bit for bit."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rot, wts, bounds, bias, ref = _setup(N, K, 2, 500 + N + K)
+    x = _acts(M, K, 31 + M)
+    t = int(bounds[1])
+    codes, scales = trdq.trdq_rotate_quantize(rot, t, to_dev_bf16(x))
+    bias_d = to_dev_bf16(bias)
+    y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
+    splits, nbytes = trdq.trdq_linear_splitk_workspace(wts, M)
+    if M >= 4096:
+        assert splits == 1 and nbytes == 0
+    else:
+        assert splits >= 2 and nbytes == splits * M * N * 4
+    ws = torch.full((max(nbytes, 16),), 0x5A, dtype=torch.uint8, device="cuda")    # stale contents must not matter
+    y2 = trdq.trdq_linear_splitk(wts, t, codes, scales, bias_d, workspace=ws)
+    assert torch.equal(y2, y)
+    y3 = trdq.trdq_linear_splitk(wts, t, codes, scales, None, workspace=ws)
+    assert torch.equal(y3, trdq.trdq_linear(wts, t, codes, scales, None))
+    if splits > 1:
+        with pytest.raises(trdq.TrdqError) as e:
+            trdq.trdq_linear_splitk(wts, t, codes, scales, bias_d, workspace=ws[:nbytes - 16])
+        assert e.value.status == 8
+    assert trdq.trdq_device_status() == 0
