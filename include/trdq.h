@@ -143,9 +143,8 @@ trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* cons
                             const int32_t M[2], const void* bias_bf16, void* const Y_bf16[2], const int64_t ldy[2],
                             void* stream);
 
-/* Split-K form of trdq_linear for problems with few rows and a long reduction (for example the
- * cross-attention K / V projections of 960 text rows with K = 4096, which give only 72 output tiles
- * for 148 SMs): the k range of Eq. 10's integer sum is cut into `splits` parts computed by different
+/* Split-K form of trdq_linear for problems with few rows and a very long reduction (K >= 8192 and
+ * fewer output tiles than half the SMs; shorter reductions are faster in one kernel): the k range of Eq. 10's integer sum is cut into `splits` parts computed by different
  * CTAs, their exact int32 partial sums go to a caller-provided workspace, and a second kernel adds
  * them and applies the epilogue.  Integer addition is associative, so the output is bit-identical to
  * trdq_linear's.  8-bit weights, one row segment.

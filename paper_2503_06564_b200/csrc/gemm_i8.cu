@@ -435,7 +435,9 @@ int splitk_choose(const trdq_weights* w, int32_t M) {
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int64_t tiles = static_cast<int64_t>((M + kTileM - 1) / kTileM) * ((w->N + 127) / 128);
   const int num_kb = w->K / kTileKBytes;
-  if (w->wbits != 8 || tiles <= 0 || tiles * 2 > sms) return 1;
+  // Measured on B200: the second kernel and its launch cost about as much as 40 k-blocks of main loop, so
+  // splitting only pays when the reduction is long (K >= 8192) and the tiles fill less than half the SMs.
+  if (w->wbits != 8 || tiles <= 0 || tiles * 2 > sms || num_kb < 64) return 1;
   int splits = static_cast<int>(sms / tiles);
   if (splits > 8) splits = 8;
   while (splits > 1 && num_kb / splits < 4) --splits;  // at least four k-blocks per range

@@ -267,10 +267,11 @@ def test_small_shapes_through_the_cta_pair_kernel():
 
 
 @pytest.mark.parametrize("M,N,K", [
-    (960, 1152, 4096),     # cross-attention K / V projection: 72 output tiles, two k ranges
-    (256, 1024, 1024),     # single-layer configuration: 16 tiles, the eight k-blocks split in two
-    (130, 272, 4608),      # ragged rows and columns, 36 k-blocks over several ranges
-    (4096, 1152, 1152),    # enough tiles: split-K declines (one range) and the call is the ordinary GEMM
+    (130, 272, 8192),      # ragged rows and columns, 64 k-blocks over eight ranges
+    (64, 1152, 16384),     # nine tiles, 128 k-blocks
+    (200, 1024, 9088),     # 71 k-blocks: the last range is shorter than the others
+    (960, 1152, 4096),     # cross-attention K / V projection: the reduction is too short to pay, one range
+    (4096, 1152, 1152),    # enough tiles: split-K declines and the call is the ordinary GEMM
 ])
 def test_linear_splitk_is_bit_identical(M, N, K):
     """Partial int32 sums from several CTAs per tile, added by a second kernel: integer addition does not
@@ -284,7 +285,7 @@ def test_linear_splitk_is_bit_identical(M, N, K):
     bias_d = to_dev_bf16(bias)
     y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
     splits, nbytes = trdq.trdq_linear_splitk_workspace(wts, M)
-    if M >= 4096:
+    if K < 8192:
         assert splits == 1 and nbytes == 0
     else:
         assert splits >= 2 and nbytes == splits * M * N * 4
