@@ -56,7 +56,8 @@ typedef enum trdq_status {
   TRDQ_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (no device, launch error, ...) */
   TRDQ_ERR_NOMEM = 8,     /* host or device allocation failed */
   TRDQ_ERR_TIMEOUT = 9,   /* a bounded device-side wait expired (see trdq_device_status) */
-  TRDQ_ERR_MISMATCH = 10  /* objects passed together were built for different K / groups */
+  TRDQ_ERR_MISMATCH = 10, /* objects passed together were built for different K / groups */
+  TRDQ_ERR_SCRATCH = 11   /* the problem needs more than the library's built-in scratch area (trdq_linear_splitk_static) */
 } trdq_status;
 
 /* Description of the per-group transforms (Time-Rotation, Sec. 3.2).  All arrays are
@@ -157,6 +158,27 @@ trdq_status trdq_linear_splitk_workspace(const trdq_weights* w, int32_t M, int32
 trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
                                const void* bias_bf16, void* Y_bf16, int64_t ldy, void* workspace, uint64_t workspace_bytes,
                                void* stream);
+
+/* trdq_linear_splitk for callers that cannot provide a workspace because they cannot allocate device
+ * memory at this point: an inference server that handed all device memory to its own pool at start-up
+ * (a cudaMalloc would simply fail), or a latency-critical loop in which the device-wide synchronisation
+ * that cudaMalloc / cudaFree imply is not acceptable.  (The paper has no counterpart; this is a
+ * deployment convenience.)  The partial sums go to a fixed array of TRDQ_STATIC_SCRATCH_ELEMS int32
+ * (8 MiB) that is part of the library image: every GPU on which the library is used holds it until the
+ * process exits.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine);
+ * inputs and outputs are the caller's as in trdq_linear.
+ *   - TRDQ_ERR_SCRATCH if splits * M * N (splits as reported by trdq_linear_splitk_workspace) exceeds
+ *     TRDQ_STATIC_SCRATCH_ELEMS; nothing is launched.  With splits == 1 the scratch is not used and the
+ *     call is trdq_linear.
+ *   - The first call on a device looks up the array's device address (once per device, with that device
+ *     current) and configures the kernels; make that first call during start-up, before any stream capture.
+ *   - All calls share the one array, and it keeps the last call's contents.  That is harmless for
+ *     calls that run one after another (every value read is written by the same call first), but two
+ *     calls that overlap on the GPU -- different streams, or concurrent host threads -- race on it:
+ *     serialise them. */
+#define TRDQ_STATIC_SCRATCH_ELEMS (2u * 1024u * 1024u)
+trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
+                                      const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
 
 /* One quantized linear layer of a denoising step: rotate + quantize X into the caller's code and
  * scale buffers, then the integer GEMM with its epilogue into Y (shapes as in the two calls above). */

@@ -116,6 +116,7 @@ const char* trdq_status_string(trdq_status s) {
     case TRDQ_ERR_NOMEM: return "out of memory";
     case TRDQ_ERR_TIMEOUT: return "bounded device-side wait expired";
     case TRDQ_ERR_MISMATCH: return "objects do not belong together";
+    case TRDQ_ERR_SCRATCH: return "problem exceeds the built-in scratch area";
   }
   return "unknown status";
 }
@@ -388,6 +389,21 @@ trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* c
   if (workspace_bytes < static_cast<uint64_t>(splits) * static_cast<uint64_t>(M) * static_cast<uint64_t>(w->N) * 4u) return TRDQ_ERR_NOMEM;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
   return launch_gemm_w8_splitk(w, g, seg, bias_bf16, splits, static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream));
+}
+
+trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
+                                      const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream) {
+  if (!w) return TRDQ_ERR_NULL;
+  if (M < 0) return TRDQ_ERR_SHAPE;
+  const int splits = M > 0 ? splitk_choose(w, M) : 1;
+  if (splits <= 1) return trdq_linear(w, t, codes, scales, M, bias_bf16, Y_bf16, ldy, stream);
+  const int g = find_group(w->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (!codes || !scales || !Y_bf16) return TRDQ_ERR_NULL;
+  if (ldy < w->N) return TRDQ_ERR_SHAPE;
+  if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16)) return TRDQ_ERR_ALIGN;
+  const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
+  return launch_gemm_w8_splitk_static(w, g, seg, bias_bf16, splits, static_cast<cudaStream_t>(stream));
 }
 
 trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes, int32_t M, int32_t* acc, int64_t ldacc, void* stream) {

@@ -489,4 +489,39 @@ trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegmen
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Split-K without any allocation: the partial sums live in a fixed array that is part of the
+// library image.  Every device that loads the library carries these 8 MiB until the process exits.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) int32_t g_static_splitk_scratch[TRDQ_STATIC_SCRATCH_ELEMS];
+
+// Device address of the array on the CURRENT device.  In host code the array's name is only a handle
+// for the runtime, not an address a kernel could use, so the address is asked for once per device
+// (with that device current) and remembered.
+static int32_t* static_scratch_address() {
+  static int32_t* cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    int32_t* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_splitk_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    cached[dev] = ptr;
+  }
+  return cached[dev];
+}
+
+trdq_status launch_gemm_w8_splitk_static(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,
+                                         cudaStream_t stream) {
+  if (static_cast<uint64_t>(splits) * static_cast<uint64_t>(seg.M) * static_cast<uint64_t>(w->N) > TRDQ_STATIC_SCRATCH_ELEMS)
+    return TRDQ_ERR_SCRATCH;
+  int32_t* scratch = static_scratch_address();
+  if (!scratch) return TRDQ_ERR_CUDA;
+  // Nothing has to be cleared: the first kernel writes every partial sum (all ranges, all rows < M, all
+  // columns < N) that the second kernel reads, so what an earlier call left behind is never seen.
+  return launch_gemm_w8_splitk(w, g, seg, bias_bf16, splits, scratch, stream);
+}
+
 }  // namespace trdq

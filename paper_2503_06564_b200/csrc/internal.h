@@ -74,6 +74,8 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
 int splitk_choose(const trdq_weights* w, int32_t M);
 trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,
                                   int32_t* workspace, cudaStream_t stream);
+trdq_status launch_gemm_w8_splitk_static(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,
+                                         cudaStream_t stream);
 // gemm_i8_2cta.cu: CTA-pair kernel; TRDQ_ERR_SHAPE means "not applicable here, use the single-CTA kernel"
 trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
                                 cudaStream_t stream);

@@ -20,14 +20,14 @@ LIB_PATH = os.path.join(_HERE, "libtrdq.so")
 OK = 0
 STATUS_NAMES = {0: "TRDQ_OK", 1: "TRDQ_ERR_NULL", 2: "TRDQ_ERR_SHAPE", 3: "TRDQ_ERR_ALIGN", 4: "TRDQ_ERR_TIMESTEP",
                 5: "TRDQ_ERR_GROUP", 6: "TRDQ_ERR_WBITS", 7: "TRDQ_ERR_CUDA", 8: "TRDQ_ERR_NOMEM", 9: "TRDQ_ERR_TIMEOUT",
-                10: "TRDQ_ERR_MISMATCH"}
+                10: "TRDQ_ERR_MISMATCH", 11: "TRDQ_ERR_SCRATCH"}
 
 EXPORTS = (
     "trdq_status_string", "trdq_version", "trdq_rotation_create", "trdq_rotation_destroy", "trdq_group_of",
     "trdq_find_group", "trdq_prepare_weights", "trdq_weights_destroy", "trdq_weights_info", "trdq_weights_view",
     "trdq_weights_export",
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
-    "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk",
+    "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
 )
 
 
@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         l.trdq_run_layers.argtypes = [C.POINTER(LayerOp), i32, i32, vp]
         l.trdq_linear_splitk_workspace.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_uint64)]
         l.trdq_linear_splitk.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp, C.c_uint64, vp]
+        l.trdq_linear_splitk_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -252,6 +253,19 @@ def trdq_linear_splitk(w: Weights, t: int, codes, scales, bias_bf16=None, out=No
     ldy = int(out.stride(0)) if M > 1 else w.N
     _check(lib().trdq_linear_splitk(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, _ptr(workspace),
                                     ws_bytes, _stream()), "trdq_linear_splitk")
+    return out
+
+
+STATIC_SCRATCH_ELEMS = 2 * 1024 * 1024
+
+
+def trdq_linear_splitk_static(w: Weights, t: int, codes, scales, bias_bf16, out):
+    """Split-K linear whose partial sums go to the library's built-in scratch array: the call allocates nothing,
+    so `out` must be passed in.  For callers that cannot allocate device memory where they call this."""
+    M = int(codes.shape[0])
+    ldy = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_linear_splitk_static(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, _stream()),
+           "trdq_linear_splitk_static")
     return out
 
 

@@ -31,11 +31,11 @@ def test_every_declared_symbol_is_exported(lib):
 def test_status_strings(lib):
     from paper_2503_06564_b200 import trdq
     seen = set()
-    for code in range(0, 11):
+    for code in range(0, 12):
         s = trdq.status_string(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 11
+    assert len(seen) == 12
     assert trdq.status_string(99) == "unknown status"
     assert lib.trdq_version() >= 100
 
