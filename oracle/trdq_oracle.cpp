@@ -26,6 +26,10 @@
 // natural output order) and the 4-bit weight storage format (two's complement
 // nibbles, even k in the low nibble, one fp32 scale per 128 consecutive k).
 //
+// The full balancing transform of Eq. 9 (second block rotation after a zigzag permutation) is restated at
+// the end of this file; its permutation convention and the Hadamard form of the second rotation are, like
+// the first rotation's, conventions the paper leaves open ("parity unpinned" by the paper).
+//
 // Build: g++ -O2 -ffp-contract=off -fopenmp -shared -fPIC (no fast-math).
 #include <cmath>
 #include <cstdint>
@@ -90,6 +94,24 @@ float quantize_span(const float* v, int n, float qmax, int8_t* q) {
     q[i] = static_cast<int8_t>(r);
   }
   return scale;
+}
+
+
+// ---- full balancing transform (Sec. 3.2, Eq. 9 / Eq. 10):  G_t(X) = (X Delta) R1 P R2 ------------
+// R1 and R2 are block rotations of the same form, diag(d) . BlockDiag(H_128) / sqrt(128), with their own
+// +-1 vectors d1, d2; P is the zigzag channel permutation, held as an index vector:
+//     (v P)[j] = v[perm[j]]            (column j of P has its single 1 in row perm[j]).
+// Row by row:  u = x o vec1;  v1 = blockWHT(u);  v2[j] = fl32(v1[perm[j]] * vec2[j]);  v3 = blockWHT(v2),
+// with vec1 = d1 * Delta * 2^-3.5 (or d1 / Delta * 2^-3.5 on the weight side) and vec2 = d2 * 2^-3.5.
+void rotate2_row(const uint16_t* row_bf16, const float* vec1, const int32_t* perm, const float* vec2, int K, float* out) {
+  std::vector<float> v1(K);
+  rotate_row(row_bf16, vec1, K, v1.data());
+  for (int c = 0; c < K; c += kBlock) {
+    float u[kBlock];
+    for (int i = 0; i < kBlock; ++i) u[i] = v1[perm[c + i]] * vec2[c + i];
+    butterfly128(u);
+    for (int i = 0; i < kBlock; ++i) out[c + i] = u[i];
+  }
 }
 
 }  // namespace
@@ -276,6 +298,80 @@ void oracle_matmul_f64(const double* A, const double* B, int M, int K, int N, do
       for (int k = 0; k < K; ++k) s += A[static_cast<int64_t>(m) * K + k] * B[static_cast<int64_t>(k) * N + n];
       C[static_cast<int64_t>(m) * N + n] = s;
     }
+}
+
+// Second-stage vector of one group: vec2[j] = fl32(d2[j] * 2^-3.5)  (d2 == nullptr means all +1).
+void oracle_second_vector(const int8_t* signs2, int K, float* vec2) {
+  for (int j = 0; j < K; ++j) vec2[j] = static_cast<float>((signs2 ? static_cast<double>(signs2[j]) : 1.0) * kHadamardNorm);
+}
+
+// Zigzag permutation (Sec. 3.2): channels sorted by magnitude, largest first, are dealt to the blocks in
+// serpentine order -- round 0 fills slot 0 of blocks 0, 1, ..., B-1, round 1 fills slot 1 of blocks B-1, ..., 0,
+// and so on -- so that no block collects only the largest or only the smallest channels.  Ties keep the
+// lower channel index first.  perm[block * 128 + slot] = source channel.
+void oracle_zigzag_permutation(const float* magnitude, int K, int32_t* perm) {
+  const int blocks = K / kBlock;
+  std::vector<int32_t> order(K);
+  for (int j = 0; j < K; ++j) order[j] = j;
+  // stable insertion-style ordering written out plainly (K is at most a few thousand)
+  for (int i = 1; i < K; ++i) {
+    const int32_t c = order[i];
+    int j = i - 1;
+    while (j >= 0 && magnitude[order[j]] < magnitude[c]) {
+      order[j + 1] = order[j];
+      --j;
+    }
+    order[j + 1] = c;
+  }
+  for (int round = 0; round < kBlock; ++round)
+    for (int i = 0; i < blocks; ++i) {
+      const int block = (round % 2 == 0) ? i : blocks - 1 - i;
+      perm[block * kBlock + round] = order[round * blocks + i];
+    }
+}
+
+// Rotated rows of the full transform in fp32 (no quantisation).
+void oracle_rotate2(const uint16_t* x_bf16, int64_t ldx, int M, int K, const float* vec1, const int32_t* perm, const float* vec2,
+                    float* v) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) rotate2_row(x_bf16 + static_cast<int64_t>(m) * ldx, vec1, perm, vec2, K, v + static_cast<int64_t>(m) * K);
+}
+
+// Full transform followed by the per-row symmetric int8 quantiser (activations, or 8-bit weights per output channel).
+void oracle_rotate2_quantize(const uint16_t* x_bf16, int64_t ldx, int M, int K, const float* vec1, const int32_t* perm,
+                             const float* vec2, int8_t* codes, float* scales) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) {
+    std::vector<float> v(K);
+    rotate2_row(x_bf16 + static_cast<int64_t>(m) * ldx, vec1, perm, vec2, K, v.data());
+    scales[m] = quantize_span(v.data(), K, 127.0f, codes + static_cast<int64_t>(m) * K);
+  }
+}
+
+// Full transform of the weight rows followed by the 4-bit quantiser (one scale per 128 consecutive k).
+void oracle_prepare2_w4(const uint16_t* w_bf16, int N, int K, const float* vec1, const int32_t* perm, const float* vec2,
+                        uint8_t* packed, float* scales) {
+  const int groups = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n) {
+    std::vector<float> v(K);
+    rotate2_row(w_bf16 + static_cast<int64_t>(n) * K, vec1, perm, vec2, K, v.data());
+    for (int kg = 0; kg < groups; ++kg) {
+      int8_t q[kBlock];
+      scales[static_cast<int64_t>(n) * groups + kg] = quantize_span(v.data() + kg * kBlock, kBlock, 7.0f, q);
+      for (int i = 0; i < kBlock; i += 2) {
+        const uint8_t lo = static_cast<uint8_t>(q[i]) & 0xF;
+        const uint8_t hi = static_cast<uint8_t>(q[i + 1]) & 0xF;
+        packed[(static_cast<int64_t>(n) * K + kg * kBlock + i) / 2] = static_cast<uint8_t>(lo | (hi << 4));
+      }
+    }
+  }
+}
+
+// Dense K x K permutation matrix of an index vector, P[perm[j]][j] = 1 (fp64 cross-check path).
+void oracle_dense_permutation(const int32_t* perm, int K, double* P) {
+  for (int64_t i = 0; i < static_cast<int64_t>(K) * K; ++i) P[i] = 0.0;
+  for (int j = 0; j < K; ++j) P[static_cast<int64_t>(perm[j]) * K + j] = 1.0;
 }
 
 int oracle_num_threads() {

@@ -168,3 +168,54 @@ def matmul_f64(A, B) -> np.ndarray:
     out = np.empty((M, N), np.float64)
     _lib().oracle_matmul_f64(_p(A), _p(B), C.c_int(M), C.c_int(K), C.c_int(N), _p(out))
     return out
+
+
+def second_vector(signs2_g, K: int) -> np.ndarray:
+    s2 = None if signs2_g is None else _c(signs2_g, np.int8)
+    out = np.empty(K, np.float32)
+    _lib().oracle_second_vector(_p(s2), C.c_int(K), _p(out))
+    return out
+
+
+def zigzag_permutation(magnitude) -> np.ndarray:
+    m = _c(magnitude, np.float32)
+    perm = np.empty(m.shape[0], np.int32)
+    _lib().oracle_zigzag_permutation(_p(m), C.c_int(m.shape[0]), _p(perm))
+    return perm
+
+
+def rotate2(x_bits, vec1, perm, vec2) -> np.ndarray:
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    v = np.empty((M, K), np.float32)
+    _lib().oracle_rotate2(_p(x), C.c_int64(K), C.c_int(M), C.c_int(K), _p(_c(vec1, np.float32)), _p(_c(perm, np.int32)),
+                          _p(_c(vec2, np.float32)), _p(v))
+    return v
+
+
+def rotate2_quantize(x_bits, vec1, perm, vec2) -> Tuple[np.ndarray, np.ndarray]:
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    codes = np.empty((M, K), np.int8)
+    scales = np.empty(M, np.float32)
+    _lib().oracle_rotate2_quantize(_p(x), C.c_int64(K), C.c_int(M), C.c_int(K), _p(_c(vec1, np.float32)), _p(_c(perm, np.int32)),
+                                   _p(_c(vec2, np.float32)), _p(codes), _p(scales))
+    return codes, scales
+
+
+def prepare2_w4(w_bits, vec1, perm, vec2) -> Tuple[np.ndarray, np.ndarray]:
+    w = _c(w_bits, np.uint16)
+    N, K = w.shape
+    packed = np.empty((N, K // 2), np.uint8)
+    scales = np.empty((N, K // 128), np.float32)
+    _lib().oracle_prepare2_w4(_p(w), C.c_int(N), C.c_int(K), _p(_c(vec1, np.float32)), _p(_c(perm, np.int32)),
+                              _p(_c(vec2, np.float32)), _p(packed), _p(scales))
+    return packed, scales
+
+
+def dense_permutation(perm) -> np.ndarray:
+    pm = _c(perm, np.int32)
+    K = pm.shape[0]
+    P = np.empty((K, K), np.float64)
+    _lib().oracle_dense_permutation(_p(pm), C.c_int(K), _p(P))
+    return P

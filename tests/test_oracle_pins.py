@@ -374,3 +374,125 @@ def test_time_step_selects_parameter_set():
     assert np.array_equal(codes[0], codes[250]) and np.array_equal(codes[250], codes[499])
     assert np.array_equal(codes[500], codes[750]) and np.array_equal(codes[750], codes[999])
     assert not np.array_equal(codes[499], codes[500])
+
+
+# --------------------------------------------------------------------------- #
+# full balancing transform (Eq. 9): second rotation after the zigzag permutation
+# --------------------------------------------------------------------------- #
+def _full_setup(K, seed, with_smooth=True):
+    rng = np.random.default_rng(seed)
+    d1 = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    d2 = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.25, 4.0, K).astype(np.float32) if with_smooth else None
+    perm = rng.permutation(K).astype(np.int32)
+    return d1, d2, smooth, perm
+
+
+def test_zigzag_is_the_serpentine_deal():
+    """Sec. 3.2: highest channel to the first block, next ones to the following blocks, direction reversing at
+    the last block.  Slot r of every block therefore holds the channels ranked r*B .. r*B+B-1, in block order
+    on even rounds and in reverse block order on odd rounds."""
+    rng = np.random.default_rng(5)
+    for K in (256, 1152):
+        B = K // 128
+        mag = rng.gamma(2.0, 1.0, K).astype(np.float32)
+        perm = O.zigzag_permutation(mag)
+        assert sorted(perm.tolist()) == list(range(K))                       # a permutation
+        rank = np.empty(K, np.int64)
+        rank[np.argsort(-mag.astype(np.float64), kind="stable")] = np.arange(K)
+        slots = rank[perm].reshape(B, 128)                                   # rank of the channel in (block, slot)
+        for r in range(128):
+            expect = np.arange(r * B, (r + 1) * B)
+            assert np.array_equal(slots[:, r], expect if r % 2 == 0 else expect[::-1])
+        # balance: block totals differ by less than the spread of single channels, unlike a contiguous deal
+        sums = mag[perm].astype(np.float64).reshape(B, 128).sum(axis=1)
+        contiguous = np.sort(mag.astype(np.float64))[::-1].reshape(B, 128).sum(axis=1)
+        assert sums.max() - sums.min() <= mag.max() - mag.min()
+        assert sums.max() - sums.min() < 0.05 * (contiguous.max() - contiguous.min())
+    # a hand-checkable case: two blocks, magnitudes descending with the channel index
+    perm = O.zigzag_permutation(np.arange(256, 0, -1).astype(np.float32))
+    assert perm[:4].tolist() == [0, 3, 4, 7] and perm[128:132].tolist() == [1, 2, 5, 6]
+
+
+def test_permutation_and_full_rotation_are_orthogonal():
+    K = 256
+    d1, d2, _, perm = _full_setup(K, 11)
+    P = O.dense_permutation(perm)
+    assert np.array_equal(P @ P.T, np.eye(K)) and np.array_equal(P.sum(axis=0), np.ones(K))
+    v = np.arange(K, dtype=np.float64)
+    assert np.array_equal(v @ P, v[perm])                                    # (v P)[j] = v[perm[j]]
+    R = O.dense_rotation(d1) @ P @ O.dense_rotation(d2)
+    assert np.abs(R @ R.T - np.eye(K)).max() < 1e-6
+
+
+def test_full_transform_invariance_fp64():
+    """Eq. 9: [(X Delta) R1 P R2] . [R2^T P^T R1^T (Delta^-1 W)] = X W."""
+    K, M, N = 256, 6, 5
+    d1, d2, smooth, perm = _full_setup(K, 12)
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((M, K))
+    W = rng.standard_normal((K, N))
+    R = O.dense_rotation(d1) @ O.dense_permutation(perm) @ O.dense_rotation(d2)
+    delta = smooth.astype(np.float64)
+    G = O.matmul_f64(X * delta, R)
+    H = O.matmul_f64(np.ascontiguousarray(R.T), W / delta[:, None])
+    ref = X @ W
+    assert np.abs(O.matmul_f64(G, H) - ref).max() <= 1e-10 * np.abs(ref).max()
+
+
+def test_rotate2_matches_dense_fp64_and_its_parts():
+    K, M = 384, 9
+    d1, d2, smooth, perm = _full_setup(K, 13)
+    x = bf16(np.random.default_rng(8).standard_normal((M, K)) * 3.0)
+    a1, _ = O.fused_vectors(d1, smooth)
+    a2 = O.second_vector(d2, K)
+    assert np.array_equal(a2, (d2.astype(np.float64) * C_NORM).astype(np.float32))
+    v = O.rotate2(x, a1, perm, a2)
+    R = O.dense_rotation(d1) @ O.dense_permutation(perm) @ O.dense_rotation(d2)
+    ref = (f32_of(x).astype(np.float64) * smooth.astype(np.float64)) @ R
+    bound = 4.0 * 128 * 2.0 ** -24 * np.abs(ref).max() * np.sqrt(128)
+    assert np.abs(v - ref).max() <= bound
+    # composition of the single-stage pieces: rotate, gather by perm, scale, rotate
+    v1 = O.rotate(x, a1)
+    v2 = (v1[:, perm] * a2[None, :]).astype(np.float32)
+    ones = np.ones(K, np.float32)
+    # feed v2 through the butterfly with a unit vector: v2 is fp32, not bf16, so compare block by block via the dense H
+    Hm = O.rotate(unit_vectors(128), np.ones(128, np.float32)).astype(np.float64)
+    ref2 = np.concatenate([v2[:, c:c + 128].astype(np.float64) @ Hm for c in range(0, K, 128)], axis=1)
+    assert np.abs(v - ref2).max() <= 128 * 2.0 ** -23 * np.abs(ref2).max()
+    codes, scales = O.rotate2_quantize(x, a1, perm, a2)
+    c2, s2 = O.quantize_rows(v)
+    assert np.array_equal(codes, c2) and np.array_equal(scales, s2)
+
+
+def test_full_transform_identity_special_case():
+    """perm = identity, d2 = +1, Delta = 1: (H/sqrt(128))^2 = I, so G(X) = X diag(d1) up to fp32 rounding."""
+    K = 256
+    rng = np.random.default_rng(2)
+    d1 = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    x = bf16(rng.standard_normal((4, K)))
+    a1, _ = O.fused_vectors(d1, None)
+    v = O.rotate2(x, a1, np.arange(K, dtype=np.int32), O.second_vector(None, K))
+    ref = f32_of(x).astype(np.float64) * d1
+    assert np.abs(v - ref).max() <= 2.0 ** -20 * np.abs(ref).max()
+
+
+def test_second_rotation_balances_blocks():
+    """Sec. 3.2: after the first rotation outliers are spread inside their block only; the zigzag permutation
+    deals strong channels over all blocks and the second rotation flattens them further."""
+    K, M = 1024, 64
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((M, K))
+    x[:, :128] *= 20.0                                  # one whole block is hot
+    xb = bf16(x)
+    d1, d2, _, _ = _full_setup(K, 14, with_smooth=False)
+    a1, _ = O.fused_vectors(d1, None)
+    v1 = O.rotate(xb, a1)
+    perm = O.zigzag_permutation(np.abs(v1).max(axis=0))
+    v3 = O.rotate2(xb, a1, perm, O.second_vector(d2, K))
+    assert np.abs(v3).max(axis=1).mean() < 0.6 * np.abs(v1).max(axis=1).mean()
+    # quantisation error of the rows drops accordingly
+    def rel_err(v):
+        q, s = O.quantize_rows(v)
+        return np.linalg.norm(q * s[:, None] - v) / np.linalg.norm(v)
+    assert rel_err(v3) < 0.7 * rel_err(v1)
