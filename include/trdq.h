@@ -85,6 +85,23 @@ const char* trdq_status_string(trdq_status s);
 trdq_status trdq_rotation_create(const trdq_rotation_spec* spec, trdq_rotation** out);
 trdq_status trdq_rotation_destroy(trdq_rotation* rot);
 
+/* Tables for the FULL balancing transform of Eq. 9 / Eq. 10,
+ *     G_t(X) = (X . Delta_t) . R1_t . P_t . R2_t,      H_t(W) = R2_t^T . P_t^T . R1_t^T . (Delta_t^-1 . W):
+ * R1 is the rotation described by `spec`, P the zigzag channel permutation given as an index vector
+ * ((v P)[j] = v[perm[j]]), and R2 a second block rotation of the same form with its own +-1 vector:
+ *   v1 = ((x o act) . BlockDiag(H_128));  v2[j] = fl32(v1[perm[j]] * fl32(d2[j] * 2^-3.5));  v3 = v2 . BlockDiag(H_128)
+ * perm: host int32 [G][K], each group a permutation of 0 .. K-1 (TRDQ_ERR_GROUP otherwise); signs2: host
+ * int8 [G][K] of +-1, or NULL for all +1.  K <= 16384.  An object created here makes trdq_rotate_quantize,
+ * trdq_prepare_weights and everything built on them use the full transform; the GEMM is unchanged. */
+trdq_status trdq_rotation_create_full(const trdq_rotation_spec* spec, const int32_t* perm, const int8_t* signs2,
+                                      trdq_rotation** out);
+
+/* Zigzag permutation of Sec. 3.2 from per-channel magnitudes (host arrays; K a multiple of 128): channels
+ * sorted by magnitude, largest first (ties: lower index first), are dealt to the K/128 blocks in serpentine
+ * order -- round r fills slot r of blocks 0 .. B-1 when r is even and of blocks B-1 .. 0 when r is odd --
+ * so strong channels are spread evenly over the blocks before the second rotation.  Pure host arithmetic. */
+trdq_status trdq_zigzag_permutation(const float* magnitude, int32_t K, int32_t* perm);
+
 /* Time-step -> group (Sec. 3.2: the parameter set is selected by the current time-step).
  * Pure host arithmetic.  TRDQ_ERR_TIMESTEP if t is outside the covered range. */
 trdq_status trdq_group_of(const trdq_rotation* rot, int32_t t, int32_t* g);

@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument validation, the time-step -> group table, object
 // lifetime, tensor-map encoding and the device status word.  No arithmetic of the method
 // happens here except the fused per-channel vectors, which are formed once per group.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -169,10 +170,65 @@ trdq_status trdq_rotation_create(const trdq_rotation_spec* spec, trdq_rotation**
   return TRDQ_OK;
 }
 
+trdq_status trdq_rotation_create_full(const trdq_rotation_spec* spec, const int32_t* perm, const int8_t* signs2, trdq_rotation** out) {
+  if (!spec || !perm || !out) return TRDQ_ERR_NULL;
+  if (spec->K <= 0 || spec->K % TRDQ_BLOCK != 0 || spec->K > 16384) return TRDQ_ERR_SHAPE;
+  if (spec->num_groups < 1) return TRDQ_ERR_GROUP;
+  const int G = spec->num_groups, K = spec->K;
+  const size_t n = static_cast<size_t>(G) * K;
+  std::vector<char> seen(K);
+  for (int g = 0; g < G; ++g) {
+    std::fill(seen.begin(), seen.end(), 0);
+    for (int j = 0; j < K; ++j) {
+      const int32_t s = perm[static_cast<size_t>(g) * K + j];
+      if (s < 0 || s >= K || seen[s]) return TRDQ_ERR_GROUP;
+      seen[s] = 1;
+    }
+  }
+  if (signs2)
+    for (size_t i = 0; i < n; ++i)
+      if (signs2[i] != 1 && signs2[i] != -1) return TRDQ_ERR_GROUP;
+  trdq_rotation* rot = nullptr;
+  const trdq_status st = trdq_rotation_create(spec, &rot);
+  if (st != TRDQ_OK) return st;
+  const double norm = 0x1.6a09e667f3bcdp-4;  // 2^-3.5
+  std::vector<float> v2(n);
+  for (size_t i = 0; i < n; ++i) v2[i] = static_cast<float>((signs2 ? static_cast<double>(signs2[i]) : 1.0) * norm);
+  if (cudaMalloc(&rot->perm, n * sizeof(int32_t)) != cudaSuccess || cudaMalloc(&rot->vec2, n * sizeof(float)) != cudaSuccess) {
+    cudaGetLastError();
+    trdq_rotation_destroy(rot);
+    return TRDQ_ERR_NOMEM;
+  }
+  if (cudaMemcpy(rot->perm, perm, n * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(rot->vec2, v2.data(), n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+    trdq_rotation_destroy(rot);
+    return TRDQ_ERR_CUDA;
+  }
+  *out = rot;
+  return TRDQ_OK;
+}
+
+trdq_status trdq_zigzag_permutation(const float* magnitude, int32_t K, int32_t* perm) {
+  if (!magnitude || !perm) return TRDQ_ERR_NULL;
+  if (K <= 0 || K % TRDQ_BLOCK != 0) return TRDQ_ERR_SHAPE;
+  const int blocks = K / TRDQ_BLOCK;
+  std::vector<int32_t> order(K);
+  for (int j = 0; j < K; ++j) order[j] = j;
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return magnitude[a] > magnitude[b]; });
+  for (int round = 0; round < TRDQ_BLOCK; ++round)
+    for (int i = 0; i < blocks; ++i) {
+      const int block = (round & 1) ? blocks - 1 - i : i;
+      perm[block * TRDQ_BLOCK + round] = order[static_cast<size_t>(round) * blocks + i];
+    }
+  return TRDQ_OK;
+}
+
 trdq_status trdq_rotation_destroy(trdq_rotation* rot) {
   if (!rot) return TRDQ_OK;
   if (rot->act_vec) cudaFree(rot->act_vec);
   if (rot->weight_vec) cudaFree(rot->weight_vec);
+  if (rot->perm) cudaFree(rot->perm);
+  if (rot->vec2) cudaFree(rot->vec2);
   delete rot;
   return TRDQ_OK;
 }
@@ -229,8 +285,12 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
       trdq_weights_destroy(w);
       return TRDQ_ERR_NOMEM;
     }
-    const cudaError_t e = launch_rotate_quantize(W_bf16, K, N, K, rot->weight_vec + static_cast<size_t>(g) * K, wbits == 8 ? 0 : 1,
-                                                 gw.codes, gw.scales, static_cast<cudaStream_t>(stream));
+    const cudaError_t e =
+        rot->perm ? launch_rotate2_quantize(W_bf16, K, N, K, rot->weight_vec + static_cast<size_t>(g) * K, rot->perm + static_cast<size_t>(g) * K,
+                                            rot->vec2 + static_cast<size_t>(g) * K, wbits == 8 ? 0 : 1, gw.codes, gw.scales,
+                                            static_cast<cudaStream_t>(stream))
+                  : launch_rotate_quantize(W_bf16, K, N, K, rot->weight_vec + static_cast<size_t>(g) * K, wbits == 8 ? 0 : 1, gw.codes,
+                                           gw.scales, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
       trdq_weights_destroy(w);
       return TRDQ_ERR_CUDA;
@@ -321,6 +381,12 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
   if (ldx < rot->K) return TRDQ_ERR_SHAPE;
   if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return TRDQ_ERR_ALIGN;
   const float* vec = rot->act_vec + static_cast<size_t>(g) * rot->K;
+  if (rot->perm) {
+    const cudaError_t e2 = launch_rotate2_quantize(X_bf16, ldx, M, rot->K, vec, rot->perm + static_cast<size_t>(g) * rot->K,
+                                                   rot->vec2 + static_cast<size_t>(g) * rot->K, 0, codes, scales,
+                                                   static_cast<cudaStream_t>(stream));
+    return e2 == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  }
   if (rotate_quantize_prefers_tma(M, rot->K))
     return launch_rotate_quantize_tma(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream));
   const cudaError_t e = launch_rotate_quantize(X_bf16, ldx, M, rot->K, vec, 0, codes, scales, static_cast<cudaStream_t>(stream));

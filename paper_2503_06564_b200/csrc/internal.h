@@ -15,6 +15,9 @@ struct trdq_rotation {
   std::vector<int32_t> t_bounds;  // host [G+1]
   float* act_vec = nullptr;       // dev [G][K]: d * Delta * 2^-3.5
   float* weight_vec = nullptr;    // dev [G][K]: d / Delta * 2^-3.5
+  // full balancing transform (Eq. 9) only; perm == nullptr means the single-rotation path
+  int32_t* perm = nullptr;        // dev [G][K]: (v P)[j] = v[perm[j]]
+  float* vec2 = nullptr;          // dev [G][K]: d2 * 2^-3.5, scaling before the second rotation
 };
 
 namespace trdq {
@@ -51,6 +54,9 @@ uint32_t* device_status_word();  // device address of the status word of the cur
 // mode 0: per-row int8 codes + fp32 scale per row; mode 1: per-128-block int4 codes packed + scale per block
 cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
                                    void* codes, float* scales, cudaStream_t stream);
+
+cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec1, const int32_t* perm,
+                                    const float* vec2, int mode, void* codes, float* scales, cudaStream_t stream);
 
 // rotate_quantize_tma.cu: per-row int8 path for rows of at most 36 blocks (TMA-staged, one thread per block)
 int rotate_quantize_tma_rows(int32_t K);  // rows per tile, 0 if K is too wide for this kernel

@@ -188,6 +188,108 @@ __global__ void __launch_bounds__(1024) rotate_quantize_kernel(const __nv_bfloat
 
 
 // ---------------------------------------------------------------------------------------------
+// Full balancing transform of Eq. 9 / Eq. 10:  (x o vec1) . R1-blocks, zigzag permutation, scale by vec2,
+// second block rotation, then the quantizer.  Same lane-group layout as the kernel above (8 lanes per
+// 128-block).  Between the two rotations the rotated row is parked in shared memory as fp32 so that every
+// lane group can gather its 128 permuted channels from anywhere in the row:
+//     v2[j] = fl32(v1[perm[j]] * vec2[j]).
+// MODE 0: int8 per row.  MODE 1: int4 per 128-block, packed.
+// ---------------------------------------------------------------------------------------------
+template <int MODE>
+__global__ void __launch_bounds__(1024) rotate2_quantize_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K,
+                                                                const float* __restrict__ vec1, const int32_t* __restrict__ perm,
+                                                                const float* __restrict__ vec2, int8_t* __restrict__ codes,
+                                                                uint8_t* __restrict__ packed, float* __restrict__ scales,
+                                                                int32_t rows_per_tile) {
+  extern __shared__ float row_buf[];  // [rows_per_tile][K]
+  __shared__ unsigned int row_max[3][32];
+  const int nb = K / TRDQ_BLOCK;
+  const int lane8 = threadIdx.x & (kLanesPerBlock - 1);
+  const int group = threadIdx.x / kLanesPerBlock;
+  const bool active = group < rows_per_tile * nb;
+  const int r = active ? group / nb : 0;
+  const int b = active ? group % nb : 0;
+  const int col0 = b * TRDQ_BLOCK + lane8 * kElemsPerLane;
+
+  if (threadIdx.x < 32) row_max[0][threadIdx.x] = 0u;
+  float v1reg[16], v2reg[16];
+  int src[16];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float4 f = __ldg(reinterpret_cast<const float4*>(vec1 + col0) + j);
+    const float4 g2 = __ldg(reinterpret_cast<const float4*>(vec2 + col0) + j);
+    const int4 pi = __ldg(reinterpret_cast<const int4*>(perm + col0) + j);
+    v1reg[4 * j] = f.x, v1reg[4 * j + 1] = f.y, v1reg[4 * j + 2] = f.z, v1reg[4 * j + 3] = f.w;
+    v2reg[4 * j] = g2.x, v2reg[4 * j + 1] = g2.y, v2reg[4 * j + 2] = g2.z, v2reg[4 * j + 3] = g2.w;
+    src[4 * j] = pi.x, src[4 * j + 1] = pi.y, src[4 * j + 2] = pi.z, src[4 * j + 3] = pi.w;
+  }
+  __syncthreads();
+
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  int it = 0;
+  for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    const int buf = it % 3;
+    if (threadIdx.x < 32) row_max[(it + 1) % 3][threadIdx.x] = 0u;
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    const bool valid = active && row < M;
+
+    float u[16];
+    if (valid) {
+      load_scaled16(reinterpret_cast<const uint4*>(x + row * ldx + col0), v1reg, u);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) u[i] = 0.0f;
+    }
+    wht128(u, lane8);  // first rotation
+    if (active) {
+      float4* dst = reinterpret_cast<float4*>(row_buf + static_cast<size_t>(r) * K + col0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dst[j] = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
+    }
+    __syncthreads();
+    // permutation (a gather over the whole row) and the second rotation's scaling
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = __fmul_rn(row_buf[static_cast<size_t>(r) * K + src[i]], v2reg[i]);
+    wht128(u, lane8);  // second rotation
+    const float gmax = group_max(absmax16(u));
+    if (MODE == 0 && valid && lane8 == 0) atomicMax(&row_max[buf][r], __float_as_uint(gmax));
+    __syncthreads();  // row maxima complete; every gather of this tile is done, the row buffer may be overwritten
+
+    if (!valid) continue;
+    const int64_t elem = row * K + col0;
+    if (MODE == 0) {
+      const float amax = __uint_as_float(row_max[buf][r]);
+      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+      uint32_t out[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          int q = quantize_one(u[4 * j + e], inv);
+          q = max(-127, min(127, q));
+          word |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * e);
+        }
+        out[j] = word;
+      }
+      *reinterpret_cast<uint4*>(codes + elem) = make_uint4(out[0], out[1], out[2], out[3]);
+      if (b == 0 && lane8 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
+    } else {
+      const float inv = gmax > 0.0f ? __fdiv_rn(7.0f, gmax) : 0.0f;
+      uint32_t out[2] = {0u, 0u};
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        int q = quantize_one(u[i], inv);
+        q = max(-7, min(7, q));
+        out[i / 8] |= (static_cast<uint32_t>(q) & 0xFu) << (4 * (i % 8));
+      }
+      *reinterpret_cast<uint2*>(packed + elem / 2) = make_uint2(out[0], out[1]);
+      if (lane8 == 0) scales[row * nb + b] = __fdiv_rn(gmax, 7.0f);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Fast path for per-row int8 codes (the online activation kernel).
 //
 // Four lanes own one 128-block of one row, 32 elements each, as four 16-byte chunks interleaved
@@ -390,6 +492,39 @@ cudaError_t dispatch(const void* x, int64_t ldx, int32_t M, int32_t K, const flo
 }
 
 }  // namespace
+
+// Full transform.  Rows of up to 128 blocks (K <= 16384); cudaErrorInvalidValue beyond that.
+cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec1, const int32_t* perm,
+                                    const float* vec2, int mode, void* codes, float* scales, cudaStream_t stream) {
+  if (M == 0) return cudaSuccess;
+  const int nb = K / TRDQ_BLOCK;
+  if (nb > 128) return cudaErrorInvalidValue;
+  int rows = 32 / nb;
+  if (rows < 1) rows = 1;
+  int threads = rows * nb * kLanesPerBlock;
+  threads = (threads + 31) / 32 * 32;
+  const size_t smem = static_cast<size_t>(rows) * K * sizeof(float);
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  static bool configured[16] = {};
+  if (dev >= 0 && dev < 16 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(rotate2_quantize_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(rotate2_quantize_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  const int num_tiles = (M + rows - 1) / rows;
+  const int ctas_per_sm = max(1, min(2048 / threads, static_cast<int>((200 * 1024) / (smem + 1024))));
+  const int grid = min(num_tiles, sms * ctas_per_sm);
+  if (mode == 0)
+    rotate2_quantize_kernel<0><<<grid, threads, smem, stream>>>(static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec1, perm, vec2,
+                                                                static_cast<int8_t*>(codes), static_cast<uint8_t*>(codes), scales, rows);
+  else
+    rotate2_quantize_kernel<1><<<grid, threads, smem, stream>>>(static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec1, perm, vec2,
+                                                                static_cast<int8_t*>(codes), static_cast<uint8_t*>(codes), scales, rows);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,
                                    void* codes, float* scales, cudaStream_t stream) {

@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--full-transform", action="store_true", help="rq: rotation, zigzag permutation, second rotation (Eq. 9)")
     ap.add_argument("--splitk", action="store_true", help="gemm: use trdq_linear_splitk with a preallocated workspace")
     ap.add_argument("--no-graph", action="store_true", help="time individual launches issued from Python (profiler runs)")
     args = ap.parse_args()
@@ -35,7 +36,8 @@ def main():
     M, K, N = args.M, args.K, args.N
     rng = np.random.default_rng(0)
     signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
-    rot = trdq.Rotation(K, [0, 1000], signs, None)
+    perm = rng.permutation(K).astype(np.int32)[None, :] if args.full_transform else None
+    rot = trdq.Rotation(K, [0, 1000], signs, None, perm=perm)
     xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(args.sets)]
     codes = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(args.sets)]
     scales = [torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(args.sets)]

@@ -28,6 +28,7 @@ EXPORTS = (
     "trdq_weights_export",
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
+    "trdq_rotation_create_full", "trdq_zigzag_permutation",
 )
 
 
@@ -63,6 +64,8 @@ def lib() -> C.CDLL:
         l.trdq_version.restype = C.c_int32
         vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
         l.trdq_rotation_create.argtypes = [C.POINTER(RotationSpec), C.POINTER(vp)]
+        l.trdq_rotation_create_full.argtypes = [C.POINTER(RotationSpec), C.POINTER(i32), C.POINTER(C.c_int8), C.POINTER(vp)]
+        l.trdq_zigzag_permutation.argtypes = [C.POINTER(C.c_float), i32, C.POINTER(i32)]
         l.trdq_rotation_destroy.argtypes = [vp]
         l.trdq_group_of.argtypes = [vp, i32, C.POINTER(i32)]
         l.trdq_find_group.argtypes = [C.POINTER(i32), i32, i32, C.POINTER(i32)]
@@ -110,10 +113,21 @@ def trdq_find_group(t_bounds: Sequence[int], t: int) -> int:
     return g.value
 
 
+def trdq_zigzag_permutation(magnitude) -> np.ndarray:
+    """Zigzag channel permutation (int32 [K]) from per-channel magnitudes; host only."""
+    m = np.ascontiguousarray(magnitude, dtype=np.float32)
+    perm = np.empty(m.shape[0], np.int32)
+    _check(lib().trdq_zigzag_permutation(m.ctypes.data_as(C.POINTER(C.c_float)), int(m.shape[0]),
+                                         perm.ctypes.data_as(C.POINTER(C.c_int32))), "trdq_zigzag_permutation")
+    return perm
+
+
 class Rotation:
     """Handle of a trdq_rotation (per-group device tables of one C_in)."""
 
-    def __init__(self, K: int, t_bounds, signs, smooth=None, block: int = 128):
+    def __init__(self, K: int, t_bounds, signs, smooth=None, block: int = 128, perm=None, signs2=None):
+        """perm (int32 [G][K]) selects the full transform of Eq. 9: rotation, zigzag permutation, second rotation
+        (signs2: its +-1 vector, int8 [G][K] or None)."""
         self._h = C.c_void_p()
         b = np.ascontiguousarray(t_bounds, dtype=np.int32)
         s = np.ascontiguousarray(signs, dtype=np.int8)
@@ -121,7 +135,14 @@ class Rotation:
         spec = RotationSpec(int(K), int(block), int(len(b) - 1), b.ctypes.data_as(C.POINTER(C.c_int32)),
                             s.ctypes.data_as(C.POINTER(C.c_int8)),
                             None if sm is None else sm.ctypes.data_as(C.POINTER(C.c_float)))
-        _check(lib().trdq_rotation_create(C.byref(spec), C.byref(self._h)), "trdq_rotation_create")
+        if perm is None:
+            _check(lib().trdq_rotation_create(C.byref(spec), C.byref(self._h)), "trdq_rotation_create")
+        else:
+            pm = np.ascontiguousarray(perm, dtype=np.int32)
+            s2 = None if signs2 is None else np.ascontiguousarray(signs2, dtype=np.int8)
+            _check(lib().trdq_rotation_create_full(C.byref(spec), pm.ctypes.data_as(C.POINTER(C.c_int32)),
+                                                   None if s2 is None else s2.ctypes.data_as(C.POINTER(C.c_int8)),
+                                                   C.byref(self._h)), "trdq_rotation_create_full")
         self.K = int(K)
         self.num_groups = int(len(b) - 1)
 

@@ -98,3 +98,21 @@ def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):
     monkeypatch.setattr(trdq, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(ImportError):
         trdq.lib()
+
+
+def test_zigzag_permutation_matches_the_oracle_and_rejects_bad_input(lib):
+    """Host-only: the library's zigzag deal equals the oracle's on random magnitudes, ties included."""
+    from oracle import trdq_oracle as O
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(0)
+    for K in (128, 256, 1152, 4608):
+        mag = rng.gamma(2.0, 1.0, K).astype(np.float32)
+        mag[rng.choice(K, K // 10, replace=False)] = mag[0]          # ties
+        assert np.array_equal(trdq.trdq_zigzag_permutation(mag), O.zigzag_permutation(mag))
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_zigzag_permutation(np.ones(100, np.float32))
+    assert e.value.status == 2
+    # a full-transform specification with a non-permutation is refused on the host
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.Rotation(256, [0, 1000], np.ones((1, 256), np.int8), perm=np.zeros((1, 256), np.int32))
+    assert e.value.status == 5
