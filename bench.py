@@ -26,6 +26,10 @@ from paper_2503_06564_b200 import workloads as WL
 
 METRIC = "rotated_w8a8_linear_tops"
 UNIT = "TOPS"
+# DRAM traffic per unit of algorithmic work, from the Nsight Compute captures summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum of one launch); None once a kernel has changed since its capture.
+GEMM_PAIR_DRAM_BYTES_PER_OP = 130.5e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
+RQ_TMA_DRAM_BYTES_PER_ALG_BYTE = 191.7 / 226.6      # rotate_quantize_tma_kernel, M = 65536, K = 1152
 INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -387,11 +391,15 @@ def run_ours(args, wl: WL.Workload):
         "gemm_tops": gemm_tops,
         "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
         "roofline": {"kernel": gemm_kernel, "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
-                     "unit": "TOPS", "frac": gemm_tops / int8_peak, "traffic": None,
+                     "unit": "TOPS", "frac": gemm_tops / int8_peak,
+                     "traffic": (GEMM_PAIR_DRAM_BYTES_PER_OP * ops / n_ops) if gemm_kernel == "gemm_w8a8_pair_kernel" else None,
+                     "traffic_note": "bytes per launch: capture at M=16384,K=1152,N=4608 scaled by the ops of an average launch of this workload",
                      "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
         "roofline_rotate_quantize": {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
-                                     "traffic": None, "peak_source": peaks["_source"]},
+                                     "traffic": RQ_TMA_DRAM_BYTES_PER_ALG_BYTE * step_rq_bytes(wl) / n_ops,
+                                     "traffic_note": "bytes per launch: TMA-kernel capture at M=65536,K=1152 scaled by algorithmic bytes",
+                                     "peak_source": peaks["_source"]},
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},
         "gpu_launches": 2 * n_ops * args.steps,
