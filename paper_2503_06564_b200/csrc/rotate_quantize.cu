@@ -315,6 +315,46 @@ __device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
   return __byte_perm(lo, hi, 0x5410);
 }
 
+// 128-point transform of one block spread over four lanes (16 fp32 pairs per lane, layout as described above).
+__device__ __forceinline__ void wht128_lanes4(float2 (&v)[16], int lane4) {
+  // h = 1: inside a pair
+#pragma unroll
+  for (int p = 0; p < 16; ++p) v[p] = make_float2(__fadd_rn(v[p].x, v[p].y), __fsub_rn(v[p].x, v[p].y));
+  // h = 2, 4: pair index bits 0, 1
+#pragma unroll
+  for (int hb = 1; hb <= 2; hb <<= 1) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if ((p & hb) == 0) {
+        const float2 a = v[p], c2 = v[p + hb];
+        v[p] = __fadd2_rn(a, c2);
+        v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+      }
+    }
+  }
+  // h = 8, 16: lanes l ^ 1, l ^ 2; upper lane computes other - own, lower lane own + other
+#pragma unroll
+  for (int mask = 1; mask <= 2; mask <<= 1) {
+    const float sgn = (lane4 & mask) ? -1.0f : 1.0f;
+    const float2 s2 = make_float2(sgn, sgn);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) v[p] = __ffma2_rn(v[p], s2, shfl_xor2(v[p], mask));
+  }
+  // h = 32, 64: pair index bits 2, 3 (the chunk of the lane)
+#pragma unroll
+  for (int hb = 4; hb <= 8; hb <<= 1) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if ((p & hb) == 0) {
+        const float2 a = v[p], c2 = v[p + hb];
+        v[p] = __fadd2_rn(a, c2);
+        v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+      }
+    }
+  }
+
+}
+
 template <int MIN_CTAS>
 __global__ void __launch_bounds__(320, MIN_CTAS)
 rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K, const float* __restrict__ vec,
@@ -372,41 +412,7 @@ rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, in
     }
     fetch(tile + gridDim.x);  // next tile's rows are in flight while this one is transformed
 
-    // h = 1: inside a pair
-#pragma unroll
-    for (int p = 0; p < 16; ++p) v[p] = make_float2(__fadd_rn(v[p].x, v[p].y), __fsub_rn(v[p].x, v[p].y));
-    // h = 2, 4: pair index bits 0, 1
-#pragma unroll
-    for (int hb = 1; hb <= 2; hb <<= 1) {
-#pragma unroll
-      for (int p = 0; p < 16; ++p) {
-        if ((p & hb) == 0) {
-          const float2 a = v[p], c2 = v[p + hb];
-          v[p] = __fadd2_rn(a, c2);
-          v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
-        }
-      }
-    }
-    // h = 8, 16: lanes l ^ 1, l ^ 2; upper lane computes other - own, lower lane own + other
-#pragma unroll
-    for (int mask = 1; mask <= 2; mask <<= 1) {
-      const float sgn = (lane4 & mask) ? -1.0f : 1.0f;
-      const float2 s2 = make_float2(sgn, sgn);
-#pragma unroll
-      for (int p = 0; p < 16; ++p) v[p] = __ffma2_rn(v[p], s2, shfl_xor2(v[p], mask));
-    }
-    // h = 32, 64: pair index bits 2, 3 (the chunk of the lane)
-#pragma unroll
-    for (int hb = 4; hb <= 8; hb <<= 1) {
-#pragma unroll
-      for (int p = 0; p < 16; ++p) {
-        if ((p & hb) == 0) {
-          const float2 a = v[p], c2 = v[p + hb];
-          v[p] = __fadd2_rn(a, c2);
-          v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
-        }
-      }
-    }
+    wht128_lanes4(v, lane4);
 
     float m = 0.0f;
 #pragma unroll
@@ -426,6 +432,129 @@ rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, in
       // the assembler, so the product is written as fma(v, inv, zero) with `zero` a kernel argument
       // equal to 0.0f: one rounding of v * inv, and nothing left to contract.
       const float2 zero2 = make_float2(zero, zero);
+      int8_t* dst = codes + row * K + col0;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float2 q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
+        *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
+      }
+      if (b == 0 && lane4 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
+    }
+  }
+}
+
+// Full transform (Eq. 9) in the four-lanes-per-block layout, per-row int8 codes: first rotation as above, the
+// rotated row parked in shared memory as fp32, gather by the permutation with the second scaling
+// (v2[j] = fl32(v1[perm[j]] * vec2[j])), second rotation, quantizer.  The permutation indices of a thread's
+// 32 columns do not change from tile to tile and are kept packed two per register (K <= 16384).
+template <int MIN_CTAS>
+__global__ void __launch_bounds__(320, MIN_CTAS)
+rotate2_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K, const float* __restrict__ vec1,
+                             const int32_t* __restrict__ perm, const float* __restrict__ vec2, int8_t* __restrict__ codes,
+                             float* __restrict__ scales, int32_t rows_per_tile, float zero) {
+  extern __shared__ float smem_f[];  // svec[K], then row_buf[rows_per_tile][K]
+  __shared__ unsigned int row_max[3][32];
+  float* svec = smem_f;
+  float* row_buf = smem_f + K;
+  const int nb = K / TRDQ_BLOCK;
+  const int lane4 = threadIdx.x & (kFastLanes - 1);
+  const int item = threadIdx.x / kFastLanes;
+  const bool active = item < rows_per_tile * nb;
+  const int r = active ? item / nb : 0;
+  const int b = active ? item % nb : 0;
+  const int col0 = b * TRDQ_BLOCK + lane4 * 8;
+
+  for (int i = threadIdx.x; i < K / 4; i += blockDim.x) reinterpret_cast<float4*>(svec)[i] = __ldg(reinterpret_cast<const float4*>(vec1) + i);
+  if (threadIdx.x < 32) row_max[0][threadIdx.x] = 0u;
+  uint32_t pidx[16];  // perm of columns col0 + 32c + 2j (low half) and + 1 (high half)
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int4 p0 = __ldg(reinterpret_cast<const int4*>(perm + col0 + 32 * c));
+    const int4 p1 = __ldg(reinterpret_cast<const int4*>(perm + col0 + 32 * c) + 1);
+    pidx[4 * c] = static_cast<uint32_t>(p0.x) | (static_cast<uint32_t>(p0.y) << 16);
+    pidx[4 * c + 1] = static_cast<uint32_t>(p0.z) | (static_cast<uint32_t>(p0.w) << 16);
+    pidx[4 * c + 2] = static_cast<uint32_t>(p1.x) | (static_cast<uint32_t>(p1.y) << 16);
+    pidx[4 * c + 3] = static_cast<uint32_t>(p1.z) | (static_cast<uint32_t>(p1.w) << 16);
+  }
+  __syncthreads();
+  griddep_launch_dependents();
+  griddep_wait();
+
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  const float2* sv = reinterpret_cast<const float2*>(svec + col0);
+  const float2* v2p = reinterpret_cast<const float2*>(vec2 + col0);
+  float* my_row = row_buf + static_cast<size_t>(r) * K;
+
+  uint4 raw[4];
+  auto fetch = [&](int tile) {
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    if (active && tile < num_tiles && row < M) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + col0);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) raw[c] = __ldg(src + 4 * c);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) raw[c] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  fetch(blockIdx.x);
+
+  int it = 0;
+  for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    const int buf = it % 3;
+    if (threadIdx.x < 32) row_max[(it + 1) % 3][threadIdx.x] = 0u;
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    const bool valid = active && row < M;
+
+    float2 v[16];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 xv = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+        v[4 * c + j] = __fmul2_rn(xv, sv[16 * c + j]);
+      }
+    }
+    fetch(tile + gridDim.x);
+    wht128_lanes4(v, lane4);  // first rotation
+    if (active) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float4* dst = reinterpret_cast<float4*>(my_row + col0 + 32 * c);
+        dst[0] = make_float4(v[4 * c].x, v[4 * c].y, v[4 * c + 1].x, v[4 * c + 1].y);
+        dst[1] = make_float4(v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 3].x, v[4 * c + 3].y);
+      }
+    }
+    __syncthreads();
+    // zigzag permutation (a gather over the row) and the scaling of the second rotation
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t pp = pidx[4 * c + j];
+        const float2 g2 = make_float2(my_row[pp & 0xFFFFu], my_row[pp >> 16]);
+        v[4 * c + j] = __fmul2_rn(g2, __ldg(v2p + 16 * c + j));
+      }
+    }
+    wht128_lanes4(v, lane4);  // second rotation
+
+    float m = 0.0f;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    if (valid && lane4 == 0) atomicMax(&row_max[buf][r], __float_as_uint(m));
+    __syncthreads();  // row maxima complete; all gathers done, the row buffer may be overwritten
+
+    if (valid) {
+      const float amax = __uint_as_float(row_max[buf][r]);
+      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+      const float2 inv2 = make_float2(inv, inv);
+      const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
+      const float2 zero2 = make_float2(zero, zero);  // see rotate_quantize_rows_kernel: keeps the product separately rounded
       int8_t* dst = codes + row * K + col0;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -499,6 +628,27 @@ cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, 
   if (M == 0) return cudaSuccess;
   const int nb = K / TRDQ_BLOCK;
   if (nb > 128) return cudaErrorInvalidValue;
+  if (mode == 0 && nb <= 72) {
+    // four lanes per block, packed arithmetic: about 72 lane groups per CTA, two CTAs per SM
+    int rows2 = 72 / nb;
+    if (rows2 > 32) rows2 = 32;
+    int threads2 = rows2 * nb * kFastLanes;
+    threads2 = (threads2 + 31) / 32 * 32;
+    const size_t smem2 = (static_cast<size_t>(K) + static_cast<size_t>(rows2) * K) * sizeof(float);
+    int dev2 = 0, sms2 = 148;
+    cudaGetDevice(&dev2);
+    cudaDeviceGetAttribute(&sms2, cudaDevAttrMultiProcessorCount, dev2);
+    static bool configured2[16] = {};
+    if (dev2 >= 0 && dev2 < 16 && !configured2[dev2]) {
+      const cudaError_t e = cudaFuncSetAttribute(rotate2_quantize_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e != cudaSuccess) return e;
+      configured2[dev2] = true;
+    }
+    const int tiles2 = (M + rows2 - 1) / rows2;
+    return launch_overlapped(rotate2_quantize_rows_kernel<2>, dim3(min(tiles2, sms2 * 2)), dim3(threads2), smem2, stream,
+                             static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec1, perm, vec2, static_cast<int8_t*>(codes), scales,
+                             rows2, 0.0f);
+  }
   int rows = 32 / nb;
   if (rows < 1) rows = 1;
   int threads = rows * nb * kLanesPerBlock;
