@@ -21,7 +21,7 @@
 //
 // Parity notes.  The quantizer, the integer GEMM and the dequantising epilogue are
 // pinned by the tests against closed forms and brute force.  Two things are
-// conventions of this build that the paper does not fix ("parity unpinned" by the
+// conventions of this implementation that the paper does not fix ("parity unpinned" by the
 // paper): the order of the fp32 additions inside the butterfly (h = 1, 2, ..., 64,
 // natural output order) and the 4-bit weight storage format (two's complement
 // nibbles, even k in the low nibble, one fp32 scale per 128 consecutive k).
