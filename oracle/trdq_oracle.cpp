@@ -114,6 +114,32 @@ void rotate2_row(const uint16_t* row_bf16, const float* vec1, const int32_t* per
   }
 }
 
+
+// Asymmetric 8-bit quantizer of Eq. 1-3 over `n` values, literally:  X_int = clamp(round(X / s) + z, 0, 255),
+// s = (max - min) / 255, with the zero point taken as z = -round(min / s) (Eq. 3 prints +round(min / s), which
+// with Eq. 1's "+ z" would map the minimum to 2 * min / s instead of 0; the sign is read as a typo).
+// As in the symmetric form, X / s is evaluated as X * fl(255 / (max - min)).  z is not clamped; codes are.
+// Returns the scale, writes the zero point and unsigned codes.  A constant span (max == min) has scale 0, z = 0, codes 0.
+float quantize_span_asym(const float* v, int n, uint8_t* q, int32_t* zero_point) {
+  float vmin = v[0], vmax = v[0];
+  for (int i = 1; i < n; ++i) {
+    vmin = std::fmin(vmin, v[i]);
+    vmax = std::fmax(vmax, v[i]);
+  }
+  const float range = vmax - vmin;
+  const float scale = range / 255.0f;
+  const float inv = range > 0.0f ? 255.0f / range : 0.0f;
+  const int z = -static_cast<int>(std::nearbyintf(vmin * inv));
+  for (int i = 0; i < n; ++i) {
+    int r = static_cast<int>(std::nearbyintf(v[i] * inv)) + z;
+    if (r > 255) r = 255;
+    if (r < 0) r = 0;
+    q[i] = static_cast<uint8_t>(r);
+  }
+  *zero_point = z;
+  return scale;
+}
+
 }  // namespace
 
 extern "C" {
@@ -372,6 +398,43 @@ void oracle_prepare2_w4(const uint16_t* w_bf16, int N, int K, const float* vec1,
 void oracle_dense_permutation(const int32_t* perm, int K, double* P) {
   for (int64_t i = 0; i < static_cast<int64_t>(K) * K; ++i) P[i] = 0.0;
   for (int j = 0; j < K; ++j) P[static_cast<int64_t>(perm[j]) * K + j] = 1.0;
+}
+
+// ---- literal asymmetric activations (Eq. 1-3) ------------------------------------------------------------
+// Per-row asymmetric quantiser on already-rotated fp32 rows.
+void oracle_quantize_rows_asym(const float* v, int M, int K, uint8_t* codes, float* scales, int32_t* zero_points) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    scales[m] = quantize_span_asym(v + static_cast<int64_t>(m) * K, K, codes + static_cast<int64_t>(m) * K, zero_points + m);
+}
+
+// Rotate (single block rotation, as oracle_rotate_quantize) then quantise each token with its own min / max.
+void oracle_rotate_quantize_asym(const uint16_t* x_bf16, int64_t ldx, int M, int K, const float* act_vec, uint8_t* codes,
+                                 float* scales, int32_t* zero_points) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) {
+    std::vector<float> v(K);
+    rotate_row(x_bf16 + static_cast<int64_t>(m) * ldx, act_vec, K, v.data());
+    scales[m] = quantize_span_asym(v.data(), K, codes + static_cast<int64_t>(m) * K, zero_points + m);
+  }
+}
+
+// Linear layer on asymmetric activation codes and symmetric per-channel weights, row subset:
+//   y = sx[m] * sw[n] * sum_k (q[m,k] - z[m]) * qw[n,k] + bias[n]      (integer sum exact; the rest in double, rounded once)
+void oracle_linear_asym_rows(const uint8_t* q, const float* sx, const int32_t* z, const int8_t* qw, const float* sw,
+                             const uint16_t* bias_bf16, const int64_t* rows, int num_rows, int N, int K, float* y) {
+#pragma omp parallel for schedule(static)
+  for (int i = 0; i < num_rows; ++i) {
+    const int64_t m = rows[i];
+    for (int n = 0; n < N; ++n) {
+      int64_t s = 0;
+      for (int k = 0; k < K; ++k)
+        s += (static_cast<int64_t>(q[m * K + k]) - z[m]) * static_cast<int64_t>(qw[static_cast<int64_t>(n) * K + k]);
+      double r = static_cast<double>(s) * static_cast<double>(sx[m]) * static_cast<double>(sw[n]);
+      if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      y[static_cast<int64_t>(i) * N + n] = static_cast<float>(r);
+    }
+  }
 }
 
 int oracle_num_threads() {

@@ -219,3 +219,37 @@ def dense_permutation(perm) -> np.ndarray:
     P = np.empty((K, K), np.float64)
     _lib().oracle_dense_permutation(_p(pm), C.c_int(K), _p(P))
     return P
+
+
+def quantize_rows_asym(v) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    v = _c(v, np.float32)
+    M, K = v.shape
+    codes = np.empty((M, K), np.uint8)
+    scales = np.empty(M, np.float32)
+    zp = np.empty(M, np.int32)
+    _lib().oracle_quantize_rows_asym(_p(v), C.c_int(M), C.c_int(K), _p(codes), _p(scales), _p(zp))
+    return codes, scales, zp
+
+
+def rotate_quantize_asym(x_bits, act_vec) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    codes = np.empty((M, K), np.uint8)
+    scales = np.empty(M, np.float32)
+    zp = np.empty(M, np.int32)
+    _lib().oracle_rotate_quantize_asym(_p(x), C.c_int64(K), C.c_int(M), C.c_int(K), _p(_c(act_vec, np.float32)), _p(codes),
+                                       _p(scales), _p(zp))
+    return codes, scales, zp
+
+
+def linear_asym_rows(q, sx, zp, qw, sw, bias_bits, rows) -> np.ndarray:
+    q = _c(q, np.uint8)
+    qw = _c(qw, np.int8)
+    rows = _c(rows, np.int64)
+    K = q.shape[1]
+    N = qw.shape[0]
+    b = None if bias_bits is None else _c(bias_bits, np.uint16)
+    y = np.empty((rows.size, N), np.float32)
+    _lib().oracle_linear_asym_rows(_p(q), _p(_c(sx, np.float32)), _p(_c(zp, np.int32)), _p(qw), _p(_c(sw, np.float32)), _p(b),
+                                   _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), _p(y))
+    return y

@@ -496,3 +496,63 @@ def test_second_rotation_balances_blocks():
         q, s = O.quantize_rows(v)
         return np.linalg.norm(q * s[:, None] - v) / np.linalg.norm(v)
     assert rel_err(v3) < 0.7 * rel_err(v1)
+
+
+# --------------------------------------------------------------------------- #
+# literal asymmetric quantizer (Eq. 1-3)
+# --------------------------------------------------------------------------- #
+def test_asymmetric_quantizer_eq1_to_eq3():
+    rng = np.random.default_rng(31)
+    v = (rng.standard_normal((40, 256)) * rng.uniform(0.1, 30.0, (40, 1)) + rng.uniform(-5, 5, (40, 1))).astype(np.float32)
+    q, s, z = O.quantize_rows_asym(v)
+    assert q.dtype == np.uint8
+    rng_ = v.max(axis=1) - v.min(axis=1)
+    assert np.array_equal(s, (rng_ / np.float32(255.0)).astype(np.float32))               # Eq. 2
+    deq = s[:, None].astype(np.float64) * (q.astype(np.float64) - z[:, None])
+    # nearest rounding (Eq. 1): error at most half a step, plus the half step the zero point itself was rounded by
+    assert np.all(np.abs(deq - v) <= s[:, None].astype(np.float64) * (1.0 + 1e-4))
+    # the minimum maps to code 0 and the maximum to 255 (Eq. 1-3 with z = -round(min / s))
+    assert np.all(q[np.arange(40), v.argmin(axis=1)] == 0) and np.all(q[np.arange(40), v.argmax(axis=1)] == 255)
+    # z is where the real value 0 lands
+    zero_code = np.rint(0.0 * 0 + z)
+    assert np.all(np.abs(s * (zero_code - z)) == 0)
+    # a closed-form case: values 0..255 -> s = 1, z = 0, codes = values; shifted by -100: z = 100
+    ramp = np.arange(256, dtype=np.float32)[None, :]
+    q1, s1, z1 = O.quantize_rows_asym(ramp)
+    assert s1[0] == 1.0 and z1[0] == 0 and np.array_equal(q1[0], np.arange(256))
+    q2, s2, z2 = O.quantize_rows_asym(ramp - 100.0)
+    assert s2[0] == 1.0 and z2[0] == 100 and np.array_equal(q2[0], np.arange(256))
+    # ties go to the even integer: range 510 -> inv = 0.5, values 2k+1 land on halves
+    odd = np.array([[0.0, 1.0, 3.0, 5.0, 510.0]], np.float32)
+    q3, s3, z3 = O.quantize_rows_asym(odd)
+    assert s3[0] == 2.0 and z3[0] == 0 and q3[0].tolist() == [0, 0, 2, 2, 255]
+    # constant row
+    q4, s4, z4 = O.quantize_rows_asym(np.full((1, 128), 3.5, np.float32))
+    assert s4[0] == 0.0 and z4[0] == 0 and not q4.any()
+
+
+def test_asymmetric_linear_brute_force_and_accuracy():
+    rng = np.random.default_rng(32)
+    M, N, K = 6, 5, 128
+    q = rng.integers(0, 256, (M, K)).astype(np.uint8)
+    z = rng.integers(0, 256, M).astype(np.int32)
+    qw = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    sx = rng.uniform(0.01, 0.1, M).astype(np.float32)
+    sw = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    y = O.linear_asym_rows(q, sx, z, qw, sw, None, np.arange(M))
+    ref = ((q.astype(np.int64) - z[:, None]) @ qw.astype(np.int64).T).astype(np.float64) * sx[:, None] * sw[None, :]
+    assert np.allclose(y, ref, rtol=1e-6, atol=0)
+    # equals the "accumulate unsigned codes, subtract z * column sums" form used on the tensor cores
+    acc_u = q.astype(np.int64) @ qw.astype(np.int64).T
+    colsum = qw.astype(np.int64).sum(axis=1)
+    assert np.array_equal(acc_u - z[:, None] * colsum[None, :], (q.astype(np.int64) - z[:, None]) @ qw.astype(np.int64).T)
+    # on shifted activations (a positive mean, as after a GELU) the asymmetric quantizer is the more accurate one
+    K2 = 1024
+    x = WL.to_bf16_bits(np.abs(rng.standard_normal((32, K2))) + 0.5)
+    act = np.ones(K2, np.float32)
+    v = O.rotate(x, act) * 0 + WL.bf16_bits_to_f32(x)          # no rotation: quantise the raw values
+    qa, sa, za = O.quantize_rows_asym(v)
+    qs, ss = O.quantize_rows(v)
+    err_a = np.linalg.norm(sa[:, None] * (qa.astype(np.float64) - za[:, None]) - v)
+    err_s = np.linalg.norm(ss[:, None] * qs.astype(np.float64) - v)
+    assert err_a < 0.6 * err_s
