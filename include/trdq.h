@@ -197,6 +197,21 @@ trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* c
 trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
                                       const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
 
+/* The quantizer of Eq. 1-3 taken literally for the activations (asymmetric, unsigned 8 bit, one zero point per
+ * token), after the same block rotation as trdq_rotate_quantize:
+ *   s[m] = (max - min) / 255,  z[m] = -rne(min * fl(255 / (max - min))),  q[m,k] = clamp(rne(v * fl(255 / (max - min))) + z[m], 0, 255)
+ * (Eq. 3's printed sign of z is read as a typo: with Eq. 1's "+ z" the minimum must map to code 0.)  Dequantized
+ * value: s[m] * (q - z[m]).  codes: dev uint8 [M, K]; scales: dev fp32 [M]; zero_points: dev int32 [M].
+ * K <= 10240; single rotation only (not with trdq_rotation_create_full).
+ * trdq_linear_asym consumes them with 8-bit weights:
+ *   y[m,n] = bf16( s[m] * sw[n] * (sum_k q[m,k] * qw[n,k] - z[m] * sum_k qw[n,k]) + bias[n] )
+ * the first sum on the tensor cores (unsigned x signed 8 bit), the column sums of the weight codes taken once at
+ * trdq_prepare_weights.  K <= 32768 keeps every intermediate inside int32. */
+trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M,
+                                      uint8_t* codes, float* scales, int32_t* zero_points, void* stream);
+trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
+                             int32_t M, const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
+
 /* One quantized linear layer of a denoising step: rotate + quantize X into the caller's code and
  * scale buffers, then the integer GEMM with its epilogue into Y (shapes as in the two calls above). */
 typedef struct trdq_layer_op {

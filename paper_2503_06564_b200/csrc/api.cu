@@ -308,6 +308,17 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
         return TRDQ_ERR_CUDA;
       }
     }
+    if (wbits == 8) {
+      if (cudaMalloc(&gw.colsum, static_cast<size_t>(N) * sizeof(int32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_NOMEM;
+      }
+      if (launch_weight_colsum(static_cast<const int8_t*>(gw.codes), N, K, gw.colsum, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_CUDA;
+      }
+    }
     if (wbits == 4) {
       const int n_pad = (N + 127) / 128 * 128;
       const int groups = K / TRDQ_BLOCK;
@@ -332,6 +343,7 @@ trdq_status trdq_weights_destroy(trdq_weights* w) {
   for (auto& gw : w->groups) {
     if (gw.codes) cudaFree(gw.codes);
     if (gw.scales) cudaFree(gw.scales);
+    if (gw.colsum) cudaFree(gw.colsum);
     if (gw.mult_t) cudaFree(gw.mult_t);
     if (gw.base) cudaFree(gw.base);
   }
@@ -470,6 +482,39 @@ trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const in
   if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16)) return TRDQ_ERR_ALIGN;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
   return launch_gemm_w8_splitk_static(w, g, seg, bias_bf16, splits, static_cast<cudaStream_t>(stream));
+}
+
+trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, uint8_t* codes,
+                                      float* scales, int32_t* zero_points, void* stream) {
+  if (!rot) return TRDQ_ERR_NULL;
+  if (M < 0 || rot->K > 10240 || rot->perm) return TRDQ_ERR_SHAPE;
+  const int g = find_group(rot->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (M == 0) return TRDQ_OK;
+  if (!X_bf16 || !codes || !scales || !zero_points) return TRDQ_ERR_NULL;
+  if (ldx < rot->K) return TRDQ_ERR_SHAPE;
+  if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u) ||
+      (reinterpret_cast<uintptr_t>(zero_points) & 3u))
+    return TRDQ_ERR_ALIGN;
+  const cudaError_t e = launch_rotate_quantize_asym(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, codes, scales,
+                                                    zero_points, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
+                             int32_t M, const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream) {
+  if (!w) return TRDQ_ERR_NULL;
+  if (w->wbits != 8) return TRDQ_ERR_WBITS;
+  if (M < 0 || w->K > 32768) return TRDQ_ERR_SHAPE;
+  const int g = find_group(w->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (M == 0) return TRDQ_OK;
+  if (!codes || !scales || !zero_points || !Y_bf16) return TRDQ_ERR_NULL;
+  if (ldy < w->N) return TRDQ_ERR_SHAPE;
+  if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16)) return TRDQ_ERR_ALIGN;
+  GemmSegment seg[2] = {GemmSegment{reinterpret_cast<const int8_t*>(codes), scales, Y_bf16, ldy, M}, GemmSegment{nullptr, nullptr, nullptr, ldy, 0}};
+  const int32_t* zp[2] = {zero_points, nullptr};
+  return launch_gemm_w8_asym(w, g, seg, zp, bias_bf16, static_cast<cudaStream_t>(stream));
 }
 
 trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes, int32_t M, int32_t* acc, int64_t ldacc, void* stream) {

@@ -43,7 +43,7 @@ struct Cfg {
   static constexpr int kStageBytes = kABytes + kBBytes;
   // parameters staged for the epilogue: (sw, bias) and the cancellation threshold per column, one
   // buffer per accumulator stage
-  static constexpr int kParamBytes = 2 * BN * 12;
+  static constexpr int kParamBytes = 2 * BN * 16;  // (sw, bias), threshold and (asymmetric mode) weight column sums
   static constexpr int kBarrierBytes = 256;
   // output staging: one 32-row x 32-column bf16 tile (2 KB, 64-byte swizzle) per epilogue warp
   static constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 2048;
@@ -64,6 +64,9 @@ struct alignas(64) GemmParams {
   int32_t tiles_m[2];
   const float* sw;
   const __nv_bfloat16* bias;
+  // asymmetric activation codes (mode 2): per-row zero points of each segment and per-channel sums of the weight codes
+  const int32_t* zp[2];
+  const int32_t* colsum;
   int32_t N, K, tiles_n;
   // split-K (raw-accumulator mode only): the k-blocks are cut into `splits` ranges of `kb_per_split`; split s
   // writes its partial sums at out + s * split_stride (elements).  splits = 1 is the ordinary GEMM.
@@ -91,6 +94,7 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
 }
 
 // MODE 0: bf16 dequantizing epilogue.  MODE 1: raw int32 accumulators.
+// MODE 2: unsigned activation codes with zero points (Eq. 1-3): acc - z[m] * colsum[n], then the epilogue of mode 0.
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<BN>;
@@ -168,7 +172,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
     // -------------------------------------------------------------- MMA issuer
     if (elect_one()) {
       BoundedWaiter w(p.status, kStatusTimeoutMma);
-      constexpr uint32_t idesc = umma_idesc_s8(BN);
+      constexpr uint32_t idesc = MODE == 2 ? umma_idesc_u8s8(BN) : umma_idesc_s8(BN);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -218,13 +222,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
       const TileCoord tc = tile_coord(p, tile, BN);
       float2* pb = param_buf + acc * BN;                                           // (sw, bias)
       float* thr = reinterpret_cast<float*>(param_buf + 2 * BN) + acc * BN;        // 2^-10 * |bias|
-      if (MODE == 0) {
+      int32_t* csum = reinterpret_cast<int32_t*>(reinterpret_cast<float*>(param_buf + 2 * BN) + 2 * BN) + acc * BN;
+      if (MODE != 1) {
         stage_column_params(pb, thr, p.sw, p.bias, tc.n0, p.N, BN, et, kEpilogueThreads);
+        if (MODE == 2)
+          for (int c = et; c < BN; c += kEpilogueThreads) csum[c] = tc.n0 + c < p.N ? __ldg(p.colsum + tc.n0 + c) : 0;
         asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
       }
       const int row = tc.m0 + q * 32 + lane;
       const bool row_ok = row < p.M[tc.seg];
-      const float sxm = (MODE == 0 && row_ok) ? __ldg(p.sx[tc.seg] + row) : 0.0f;
+      const float sxm = (MODE != 1 && row_ok) ? __ldg(p.sx[tc.seg] + row) : 0.0f;
+      const int32_t zrow = (MODE == 2 && row_ok) ? __ldg(p.zp[tc.seg] + row) : 0;
 
       w.wait(bar_tfull + 8 * acc, acc_phase);
       __syncwarp();
@@ -237,7 +245,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
         const int n_base = tc.n0 + c * 32;
-        if (MODE == 0) {
+        if (MODE == 2) {
+          // sum_k (q - z) * qw = sum_k q * qw - z * sum_k qw
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = static_cast<uint32_t>(static_cast<int32_t>(r[j]) - zrow * csum[c * 32 + j]);
+        }
+        if (MODE != 1) {
           const float4* pb4 = reinterpret_cast<const float4*>(pb + c * 32);
           const float4* thr4 = reinterpret_cast<const float4*>(thr + c * 32);
           uint32_t packed[16];
@@ -272,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
         acc_phase ^= 1;
       }
     }
-    if (MODE == 0 && lane == 0) bulk_wait_group<0>();  // every output tile has been written
+    if (MODE != 1 && lane == 0) bulk_wait_group<0>();  // every output tile has been written
     w.settle();
   }
 
@@ -318,14 +331,15 @@ int choose_tile_n(int64_t tiles_m, int N, int sms) {
 
 }  // namespace
 
-trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
-                           cudaStream_t stream) {
+static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, int mode,
+                                       const int32_t* const zp[2], cudaStream_t stream) {
+  const bool raw_i32 = mode == 1;
   // Large problems go to the CTA-pair kernel (two SMs per 256-row tile, a third less operand traffic per SM).
   static const int pair_min_rows = [] {
     const char* e = getenv("TRDQ_PAIR_MIN_M");
     return e ? atoi(e) : 2048;
   }();
-  if (!raw_i32 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows) {
+  if (mode == 0 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows) {
     const trdq_status st = launch_gemm_w8_pair(w, g, seg, bias_bf16, stream);
     if (st != TRDQ_ERR_SHAPE) return st;
   }
@@ -369,6 +383,9 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
   p.splits = 1;
   p.kb_per_split = w->K / kTileKBytes;
   p.split_stride = 0;
+  p.zp[0] = zp ? zp[0] : nullptr;
+  p.zp[1] = zp ? zp[1] : nullptr;
+  p.colsum = w->groups[g].colsum;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   const int64_t total = tiles_m * p.tiles_n;
@@ -377,10 +394,48 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
   cudaError_t e;
   if (raw_i32) {
     e = bn == 128 ? launch_one<128, 1>(p, grid, stream) : bn == 192 ? launch_one<192, 1>(p, grid, stream) : launch_one<256, 1>(p, grid, stream);
+  } else if (mode == 2) {
+    e = bn == 128 ? launch_one<128, 2>(p, grid, stream) : bn == 192 ? launch_one<192, 2>(p, grid, stream) : launch_one<256, 2>(p, grid, stream);
   } else {
     e = bn == 128 ? launch_one<128, 0>(p, grid, stream) : bn == 192 ? launch_one<192, 0>(p, grid, stream) : launch_one<256, 0>(p, grid, stream);
   }
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
+trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
+                           cudaStream_t stream) {
+  return launch_gemm_w8_mode(w, g, seg, bias_bf16, raw_i32 ? 1 : 0, nullptr, stream);
+}
+
+// Unsigned activation codes with per-row zero points (Eq. 1-3); `w` must carry the column sums of its codes.
+trdq_status launch_gemm_w8_asym(const trdq_weights* w, int g, const GemmSegment seg[2], const int32_t* const zp[2],
+                                const void* bias_bf16, cudaStream_t stream) {
+  if (!w->groups[g].colsum) return TRDQ_ERR_WBITS;
+  return launch_gemm_w8_mode(w, g, seg, bias_bf16, 2, zp, stream);
+}
+
+// Row sums of the int8 weight codes, one warp per output channel.
+namespace {
+__global__ void weight_colsum_kernel(const int8_t* __restrict__ codes, int32_t N, int32_t K, int32_t* __restrict__ colsum) {
+  const int n = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5);
+  if (n >= N) return;
+  const int lane = threadIdx.x & 31;
+  const int4* row = reinterpret_cast<const int4*>(codes + static_cast<int64_t>(n) * K);
+  int32_t s = 0;
+  for (int i = lane; i < K / 16; i += 32) {
+    const int4 v = row[i];
+    const int32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) s = __dp4a(wd[j], 0x01010101, s);  // four signed bytes times 1
+  }
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) colsum[n] = s;
+}
+}  // namespace
+
+cudaError_t launch_weight_colsum(const int8_t* codes, int32_t N, int32_t K, int32_t* colsum, cudaStream_t stream) {
+  weight_colsum_kernel<<<(N + 7) / 8, 256, 0, stream>>>(codes, N, K, colsum);
+  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -467,6 +522,8 @@ trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegmen
   p.tmap_b = w->groups[g].tmap_b[0];             // 128-column tiles
   p.sw = nullptr;
   p.bias = nullptr;
+  p.zp[0] = p.zp[1] = nullptr;
+  p.colsum = nullptr;
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + 127) / 128;

@@ -33,6 +33,7 @@ struct GroupWeights {
   CUtensorMap tmap_b_half[kNumTileN];   // 8-bit only: boxes of half a tile width (64 / 96 / 128 rows) for the CTA-pair kernel
   // 4-bit weights only: the scales of an output channel as integers on a common power-of-two grid,
   //   scales[n][kg] = mult_t[kg][n] * base[n]   (exact whenever the exponents of a channel span < 7 bits)
+  int32_t* colsum = nullptr;            // 8-bit only: dev int32 [N], sum over k of the codes (for asymmetric activations)
   int32_t* mult_t = nullptr;            // dev int32 [K/128][n_pad], n_pad = N rounded up to 128
   float* base = nullptr;                // dev fp32 [n_pad], a power of two (already divided by 16, see gemm_w4a8.cu)
 };
@@ -76,6 +77,11 @@ trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2
                            cudaStream_t stream);
 trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
                            cudaStream_t stream);
+trdq_status launch_gemm_w8_asym(const trdq_weights* w, int g, const GemmSegment seg[2], const int32_t* const zp[2],
+                                const void* bias_bf16, cudaStream_t stream);
+cudaError_t launch_weight_colsum(const int8_t* codes, int32_t N, int32_t K, int32_t* colsum, cudaStream_t stream);
+cudaError_t launch_rotate_quantize_asym(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, uint8_t* codes,
+                                        float* scales, int32_t* zero_points, cudaStream_t stream);
 // split-K (8-bit weights, one segment): partial int32 sums in `workspace` (splits * M * N), then reduce + epilogue
 int splitk_choose(const trdq_weights* w, int32_t M);
 trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,

@@ -228,4 +228,9 @@ __host__ __device__ constexpr uint32_t umma_idesc_s8(int n) {
          | (static_cast<uint32_t>(128 >> 4) << 24);  // M / 16
 }
 
+// Same with UNSIGNED 8-bit A (asymmetric activation codes) and signed 8-bit B.
+__host__ __device__ constexpr uint32_t umma_idesc_u8s8(int n) {
+  return (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+}
+
 }  // namespace trdq

@@ -568,6 +568,111 @@ rotate2_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, i
   }
 }
 
+// Literal asymmetric quantizer of Eq. 1-3 after the block rotation: per row min and max,
+//   s = (max - min) / 255,  z = -rne(min * fl(255 / (max - min))),  code = min(rne(v * fl(255 / (max - min))) + z, 255)
+// (the lower clamp of Eq. 1 can never bind: rounding is monotone and z cancels the minimum's own code).
+// Same four-lanes-per-block layout and butterfly as rotate_quantize_rows_kernel; the row minimum and maximum
+// are combined through shared-memory atomics on an order-preserving integer image of the floats.
+__device__ __forceinline__ unsigned int float_order_key(float f) {
+  const unsigned int b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(unsigned int k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+template <int MIN_CTAS>
+__global__ void __launch_bounds__(320, MIN_CTAS)
+rotate_quantize_rows_asym_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int32_t M, int32_t K, const float* __restrict__ vec,
+                                 uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ zero_points,
+                                 int32_t rows_per_tile) {
+  extern __shared__ float svec[];
+  __shared__ unsigned int row_hi[3][32], row_lo[3][32];
+  const int nb = K / TRDQ_BLOCK;
+  const int lane4 = threadIdx.x & (kFastLanes - 1);
+  const int item = threadIdx.x / kFastLanes;
+  const bool active = item < rows_per_tile * nb;
+  const int r = active ? item / nb : 0;
+  const int b = active ? item % nb : 0;
+
+  for (int i = threadIdx.x; i < K / 4; i += blockDim.x) reinterpret_cast<float4*>(svec)[i] = __ldg(reinterpret_cast<const float4*>(vec) + i);
+  if (threadIdx.x < 32) {
+    row_hi[0][threadIdx.x] = 0u;
+    row_lo[0][threadIdx.x] = 0xFFFFFFFFu;
+  }
+  __syncthreads();
+  griddep_launch_dependents();
+  griddep_wait();
+
+  const int num_tiles = (M + rows_per_tile - 1) / rows_per_tile;
+  const int col0 = b * TRDQ_BLOCK + lane4 * 8;
+  const float2* sv = reinterpret_cast<const float2*>(svec + col0);
+  int it = 0;
+  for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    const int buf = it % 3;
+    if (threadIdx.x < 32) {
+      row_hi[(it + 1) % 3][threadIdx.x] = 0u;
+      row_lo[(it + 1) % 3][threadIdx.x] = 0xFFFFFFFFu;
+    }
+    const int64_t row = static_cast<int64_t>(tile) * rows_per_tile + r;
+    const bool valid = active && row < M;
+    float2 v[16];
+    if (valid) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + col0);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint4 raw = __ldg(src + 4 * c);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          v[4 * c + j] = __fmul2_rn(make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u)), sv[16 * c + j]);
+      }
+    } else {
+#pragma unroll
+      for (int p = 0; p < 16; ++p) v[p] = make_float2(0.0f, 0.0f);
+    }
+    wht128_lanes4(v, lane4);
+    float hi = v[0].x, lo = v[0].x;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      hi = fmaxf(fmaxf(hi, v[p].x), v[p].y);
+      lo = fminf(fminf(lo, v[p].x), v[p].y);
+    }
+#pragma unroll
+    for (int mask = 1; mask <= 2; mask <<= 1) {
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, mask));
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, mask));
+    }
+    if (valid && lane4 == 0) {
+      atomicMax(&row_hi[buf][r], float_order_key(hi));
+      atomicMin(&row_lo[buf][r], float_order_key(lo));
+    }
+    __syncthreads();
+    if (!valid) continue;
+    const float vmax = float_from_order_key(row_hi[buf][r]);
+    const float vmin = float_from_order_key(row_lo[buf][r]);
+    const float range = __fsub_rn(vmax, vmin);
+    const float inv = range > 0.0f ? __fdiv_rn(255.0f, range) : 0.0f;
+    const int z = -__float2int_rn(__fmul_rn(vmin, inv));
+    uint8_t* dst = codes + row * K + col0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t wd[2] = {0u, 0u};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int q0 = min(__float2int_rn(__fmul_rn(v[4 * c + j].x, inv)) + z, 255);
+        const int q1 = min(__float2int_rn(__fmul_rn(v[4 * c + j].y, inv)) + z, 255);
+        wd[j / 2] |= (static_cast<uint32_t>(q0) | (static_cast<uint32_t>(q1) << 8)) << (16 * (j & 1));
+      }
+      *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(wd[0], wd[1]);
+    }
+    if (b == 0 && lane4 == 0) {
+      scales[row] = __fdiv_rn(range, 255.0f);
+      zero_points[row] = z;
+    }
+  }
+}
+
 cudaError_t launch_rows_fast(const void* x, int64_t ldx, int32_t M, int32_t K, const float* vec, void* codes, float* scales,
                              cudaStream_t stream) {
   const int nb = K / TRDQ_BLOCK;
@@ -621,6 +726,26 @@ cudaError_t dispatch(const void* x, int64_t ldx, int32_t M, int32_t K, const flo
 }
 
 }  // namespace
+
+// Asymmetric per-row quantizer (Eq. 1-3).  Rows of up to 80 blocks (K <= 10240); cudaErrorInvalidValue beyond that.
+cudaError_t launch_rotate_quantize_asym(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, uint8_t* codes,
+                                        float* scales, int32_t* zero_points, cudaStream_t stream) {
+  if (M == 0) return cudaSuccess;
+  const int nb = K / TRDQ_BLOCK;
+  if (nb > 80) return cudaErrorInvalidValue;
+  int rows = 72 / nb;
+  if (rows < 1) rows = 1;
+  if (rows > 32) rows = 32;
+  int threads = rows * nb * kFastLanes;
+  threads = (threads + 31) / 32 * 32;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int num_tiles = (M + rows - 1) / rows;
+  return launch_overlapped(rotate_quantize_rows_asym_kernel<2>, dim3(min(num_tiles, sms * 2)), dim3(threads),
+                           static_cast<size_t>(K) * sizeof(float), stream, static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec, codes,
+                           scales, zero_points, rows);
+}
 
 // Full transform.  Rows of up to 128 blocks (K <= 16384); cudaErrorInvalidValue beyond that.
 cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec1, const int32_t* perm,

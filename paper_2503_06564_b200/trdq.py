@@ -28,7 +28,7 @@ EXPORTS = (
     "trdq_weights_export",
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
-    "trdq_rotation_create_full", "trdq_zigzag_permutation",
+    "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
 )
 
 
@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
         l.trdq_linear_splitk_workspace.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_uint64)]
         l.trdq_linear_splitk.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp, C.c_uint64, vp]
         l.trdq_linear_splitk_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
+        l.trdq_rotate_quantize_asym.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp]
+        l.trdq_linear_asym.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -287,6 +289,30 @@ def trdq_linear_splitk_static(w: Weights, t: int, codes, scales, bias_bf16, out)
     ldy = int(out.stride(0)) if M > 1 else w.N
     _check(lib().trdq_linear_splitk_static(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, _stream()),
            "trdq_linear_splitk_static")
+    return out
+
+
+def trdq_rotate_quantize_asym(rot: Rotation, t: int, X_bf16):
+    """Asymmetric per-token quantizer of Eq. 1-3: (codes uint8 [M,K], scales fp32 [M], zero points int32 [M])."""
+    import torch
+    M = int(X_bf16.shape[0])
+    codes = torch.empty((M, rot.K), dtype=torch.uint8, device=X_bf16.device)
+    scales = torch.empty((M,), dtype=torch.float32, device=X_bf16.device)
+    zp = torch.empty((M,), dtype=torch.int32, device=X_bf16.device)
+    ldx = int(X_bf16.stride(0)) if M > 1 else rot.K
+    _check(lib().trdq_rotate_quantize_asym(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(codes), _ptr(scales), _ptr(zp), _stream()),
+           "trdq_rotate_quantize_asym")
+    return codes, scales, zp
+
+
+def trdq_linear_asym(w: Weights, t: int, codes, scales, zero_points, bias_bf16=None, out=None):
+    import torch
+    M = int(codes.shape[0])
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.bfloat16, device=codes.device)
+    ldy = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_linear_asym(w._h, int(t), _ptr(codes), _ptr(scales), _ptr(zero_points), M, _ptr(bias_bf16), _ptr(out), ldy,
+                                  _stream()), "trdq_linear_asym")
     return out
 
 
