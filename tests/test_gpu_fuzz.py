@@ -1,0 +1,59 @@
+"""Seeded random shapes through the whole path (rotate + quantize, both GEMM kernels, 8- and 4-bit weights,
+with and without smoothing and bias) against the oracle: small problems, many corner combinations."""
+import numpy as np
+import pytest
+
+from oracle import trdq_oracle as O
+from paper_2503_06564_b200 import workloads as WL
+from tests.util import bf16_to_f32_np, check_output, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_problem(seed):
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(1000 + seed)
+    K = 128 * int(rng.integers(1, 13))
+    N = 16 * int(rng.integers(1, 40))
+    M = int(rng.integers(1, 420))
+    G = int(rng.integers(1, 4))
+    wbits = 4 if seed % 3 == 2 else 8
+    with_smooth = bool(rng.integers(0, 2))
+    with_bias = bool(rng.integers(0, 2))
+    signs = (rng.integers(0, 2, (G, K)) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.3, 3.0, (G, K)).astype(np.float32) if with_smooth else None
+    bounds = np.sort(rng.choice(np.arange(1, 1000), G - 1, replace=False)) if G > 1 else np.array([], np.int64)
+    bounds = np.concatenate([[0], bounds, [1000]]).astype(np.int32)
+    x = rng.standard_normal((M, K)) * rng.uniform(0.1, 5.0)
+    x[:, rng.choice(K, max(1, K // 64), replace=False)] *= 25.0
+    if M > 2:
+        x[1] = 0.0
+    x = WL.to_bf16_bits(x)
+    w = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.05)
+    bias = WL.to_bf16_bits(rng.standard_normal(N) * 0.02)
+    rot = trdq.Rotation(K, bounds, signs, smooth)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(w), wbits)
+    xd = to_dev_bf16(x)
+    bias_d = to_dev_bf16(bias) if with_bias else None
+    g = int(rng.integers(0, G))
+    t = int(rng.integers(bounds[g], bounds[g + 1]))
+    assert rot.group_of(t) == g == O.group_of(bounds, t)
+    act, wv = O.fused_vectors(signs[g], None if smooth is None else smooth[g])
+    q_ref, sx_ref = O.rotate_quantize(x, act)
+    codes, scales = trdq.trdq_rotate_quantize(rot, t, xd)
+    assert np.array_equal(codes.cpu().numpy(), q_ref) and np.array_equal(scales.cpu().numpy(), sx_ref)
+    y = trdq.trdq_linear(wts, t, codes, scales, bias_d)
+    rows = np.arange(M)
+    if wbits == 8:
+        qw_ref, sw_ref = O.prepare_w8(w, wv)
+        y_ref = O.linear_w8_rows(q_ref, sx_ref, qw_ref, sw_ref, bias if with_bias else None, rows)
+        assert np.array_equal(trdq.trdq_gemm_i32(wts, t, codes).cpu().numpy(), O.gemm_i32(q_ref, qw_ref))
+    else:
+        pk_ref, sw4_ref = O.prepare_w4(w, wv)
+        y_ref = O.linear_w4_rows(q_ref, sx_ref, pk_ref, sw4_ref, bias if with_bias else None, rows)
+    wq_dev, sw_dev = wts.view_tensors(g)
+    assert np.array_equal(wq_dev.cpu().numpy(), qw_ref if wbits == 8 else pk_ref)
+    l2, ulps = check_output(bf16_to_f32_np(y), y_ref, max_ulp=2.0, rel_l2=2e-3)
+    assert ulps <= 1.0
+    assert trdq.trdq_device_status() == 0
