@@ -246,6 +246,12 @@ trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes,
  * receives the raw bits. */
 trdq_status trdq_device_status(uint32_t* word);
 
+/* Exercises the bounded wait on purpose: launches one warp that waits on a memory barrier nothing will ever
+ * signal.  The wait expires after 20 ms, sets bit 31 of the status word and the kernel ends normally; the next
+ * trdq_device_status returns TRDQ_ERR_TIMEOUT with that bit and clears it, and the device stays fully usable.
+ * For checking that a stuck pipeline would be reported instead of hanging the GPU. */
+trdq_status trdq_selftest_wait_expiry(void* stream);
+
 /* Library version, major * 100 + minor. */
 int32_t trdq_version(void);
 

@@ -98,6 +98,19 @@ static int find_group(const std::vector<int32_t>& bounds, int32_t t) {
   return -1;
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever signals.  The wait gives up
+// after 20 ms, records its bit in the status word and the kernel returns normally.
+__global__ void selftest_wait_expiry_kernel(uint32_t* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  BoundedWaiter w(status, kStatusTimeoutSelfTest, 20000000ull);
+  w.wait(smem_u32(&bar), 0);
+}
+
 }  // namespace trdq
 
 using namespace trdq;
@@ -547,6 +560,13 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
     if (st != TRDQ_OK) return st;
   }
   return TRDQ_OK;
+}
+
+trdq_status trdq_selftest_wait_expiry(void* stream) {
+  uint32_t* status = device_status_word();
+  if (!status) return TRDQ_ERR_CUDA;
+  selftest_wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status);
+  return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
 trdq_status trdq_device_status(uint32_t* word) {

@@ -12,6 +12,7 @@ enum : uint32_t {
   kStatusTimeoutMma = 1u << 1,       // MMA issuer gave up waiting for data or a free accumulator
   kStatusTimeoutEpilogue = 1u << 2,  // epilogue gave up waiting for an accumulator
   kStatusTimeoutUnpack = 1u << 3,    // int4 unpack warps gave up waiting
+  kStatusTimeoutSelfTest = 1u << 31, // the self-test's deliberately unsignalled barrier
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -79,14 +80,16 @@ struct BoundedWaiter {
   uint32_t* status;
   uint32_t bit;
   bool dead;
-  __device__ __forceinline__ BoundedWaiter(uint32_t* s, uint32_t b) : status(s), bit(b), dead(false) {}
+  uint64_t limit_ns;
+  __device__ __forceinline__ BoundedWaiter(uint32_t* s, uint32_t b, uint64_t limit = 1000000000ull)  // one second
+      : status(s), bit(b), dead(false), limit_ns(limit) {}
   __device__ __forceinline__ void wait(uint32_t bar, uint32_t parity) {
     if (dead) return;
     if (mbar_try_wait(bar, parity)) return;
     const uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
     while (!mbar_try_wait(bar, parity)) {
-      if ((++polls & 0xFF) == 0 && global_timer_ns() - t0 > 1000000000ull) {  // one second
+      if ((++polls & 0xFF) == 0 && global_timer_ns() - t0 > limit_ns) {
         dead = true;
         atomicOr(status, bit);
         return;

@@ -29,6 +29,7 @@ EXPORTS = (
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
     "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
+    "trdq_selftest_wait_expiry",
 )
 
 
@@ -85,6 +86,7 @@ def lib() -> C.CDLL:
         l.trdq_linear_splitk_static.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_rotate_quantize_asym.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp]
         l.trdq_linear_asym.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, i64, vp]
+        l.trdq_selftest_wait_expiry.argtypes = [vp]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -359,6 +361,11 @@ def trdq_run_layers(layers: LayerList, t: int, first: int = 0, count: Optional[i
     arr = layers.array()
     ptr = C.cast(C.byref(arr, first * C.sizeof(LayerOp)), C.POINTER(LayerOp))
     _check(lib().trdq_run_layers(ptr, int(n), int(t), _stream()), "trdq_run_layers")
+
+
+def trdq_selftest_wait_expiry() -> None:
+    """Launches the kernel whose only barrier is never signalled (its wait expires after 20 ms)."""
+    _check(lib().trdq_selftest_wait_expiry(_stream()), "trdq_selftest_wait_expiry")
 
 
 def trdq_device_status() -> int:

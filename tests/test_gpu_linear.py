@@ -299,3 +299,25 @@ def test_linear_splitk_is_bit_identical(M, N, K):
             trdq.trdq_linear_splitk(wts, t, codes, scales, bias_d, workspace=ws[:nbytes - 16])
         assert e.value.status == 8
     assert trdq.trdq_device_status() == 0
+
+
+def test_an_expired_wait_is_reported_and_the_device_stays_usable():
+    """Every barrier wait in the kernels has a time limit.  The self-test kernel waits on a barrier nothing signals:
+    the wait gives up after 20 ms, the status word carries its bit, and ordinary work runs fine afterwards."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    assert trdq.trdq_device_status() == 0
+    trdq.trdq_selftest_wait_expiry()
+    word = trdq.trdq_device_status()               # synchronises
+    assert word == 1 << 31
+    assert trdq.trdq_device_status() == 0          # reading clears it
+    rot, wts, bounds, bias, ref = _setup(256, 256, 1, 9)
+    x = _acts(64, 256, 2)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, to_dev_bf16(x))
+    act, qw_ref, sw_ref = ref[0]
+    q_ref, sx_ref = O.rotate_quantize(x, act)
+    assert np.array_equal(codes.cpu().numpy(), q_ref)
+    y = trdq.trdq_linear(wts, 0, codes, scales, to_dev_bf16(bias))
+    y_ref = O.linear_w8_rows(q_ref, sx_ref, qw_ref, sw_ref, bias, np.arange(64))
+    check_output(bf16_to_f32_np(y), y_ref, max_ulp=1.0)
+    assert trdq.trdq_device_status() == 0
