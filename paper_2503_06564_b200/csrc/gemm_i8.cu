@@ -135,17 +135,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) {  // descriptors are kernel arguments: fetch them while the previous kernel may still be running
+    prefetch_tensormap(&p.tmap_a[0]);
+    prefetch_tensormap(&p.tmap_a[1]);
+    prefetch_tensormap(&p.tmap_b);
+    prefetch_tensormap(&p.tmap_out[0]);
+    prefetch_tensormap(&p.tmap_out[1]);
+  }
   griddep_launch_dependents();
   griddep_wait();  // codes, scales and weights may come from the kernel before; Y may still be read by it
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
-      prefetch_tensormap(&p.tmap_a[0]);
-      prefetch_tensormap(&p.tmap_a[1]);
-      prefetch_tensormap(&p.tmap_b);
-      prefetch_tensormap(&p.tmap_out[0]);
-      prefetch_tensormap(&p.tmap_out[1]);
       BoundedWaiter w(p.status, kStatusTimeoutProducer);
       int stage = 0;
       uint32_t phase = 0;
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
         acc_phase ^= 1;
       }
     }
-    if (MODE != 1 && lane == 0) bulk_wait_group<0>();  // every output tile has been written
+    if (MODE != 1 && lane == 0) bulk_wait_group_read<0>();  // the staging tiles have been read; the stores complete before the grid does
     w.settle();
   }
 

@@ -175,17 +175,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
   cluster_sync_all();  // the peer's barriers are initialised and its tensor memory allocated before anything is signalled
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) {  // descriptors are kernel arguments: fetch them while the previous kernel may still be running
+    prefetch_tensormap(&p.tmap_a[0]);
+    prefetch_tensormap(&p.tmap_a[1]);
+    prefetch_tensormap(&p.tmap_b);
+    prefetch_tensormap(&p.tmap_out[0]);
+    prefetch_tensormap(&p.tmap_out[1]);
+  }
   griddep_launch_dependents();
   griddep_wait();
 
   if (warp == 0) {
     // ---------------------------------------------------- TMA producer (both CTAs)
     if (elect_one()) {
-      prefetch_tensormap(&p.tmap_a[0]);
-      prefetch_tensormap(&p.tmap_a[1]);
-      prefetch_tensormap(&p.tmap_b);
-      prefetch_tensormap(&p.tmap_out[0]);
-      prefetch_tensormap(&p.tmap_out[1]);
       BoundedWaiter w(p.status, kStatusTimeoutProducer);
       const uint32_t leader_full = map_to_cta(bar_full, 0);
       int stage = 0;
@@ -301,7 +303,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
         acc_phase ^= 1;
       }
     }
-    if (lane == 0) bulk_wait_group<0>();
+    if (lane == 0) bulk_wait_group_read<0>();  // the staging tiles have been read; the stores complete before the grid does
     w.settle();
   }
 

@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
         }
       }
     }
-    if (lane == 0) bulk_wait_group<0>();
+    if (lane == 0) bulk_wait_group_read<0>();  // the staging tiles have been read; the stores complete before the grid does
     w.settle();
   }
 

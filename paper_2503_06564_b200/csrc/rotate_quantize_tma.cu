@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(MAXT + 32, MINB) rotate_quantize_tma_kernel(co
       bulk_commit_group();
     }
   }
-  if (tid == 0) bulk_wait_group<0>();
+  if (tid == 0) bulk_wait_group_read<0>();  // the staging tile has been read; the stores complete before the grid does
   w.settle();
 }
 
