@@ -437,6 +437,207 @@ void oracle_linear_asym_rows(const uint8_t* q, const float* sx, const int32_t* z
   }
 }
 
+// ---- dense block rotations (Sec. 3.2, Eq. 6-8) -----------------------------------------------------------
+// Eq. 8: R = BlockDiag(R_b1 .. R_bK), every block a dense 128 x 128 orthogonal matrix (a greedy product of
+// Eq. 6 factors, built offline).  Online side of Eq. 10 with such blocks: v = (x o Delta) . R per block.
+// The smoothing vector is folded into the rows of each block and the result is STORED IN BF16 (the format
+// the matrix is applied in):  S_b[i][j] = bf16_rne(Delta[128 b + i] * R_b[i][j]).  Because S is what is
+// applied to the activations, the weight side uses the exact inverse of S (not R^T Delta^-1), so the
+// identity (X S)(S^-1 W) = X W of Eq. 9 holds whatever the rounding did.  The storage precision is a
+// convention of this implementation ("parity unpinned" by the paper, which does not say how R is held).
+
+// Round a double to the nearest bf16 (8 significand bits), ties to even; returns the bf16 bit pattern.
+static uint16_t double_to_bf16_bits(double p) {
+  if (p == 0.0) return 0;
+  int e = 0;
+  const double m = std::frexp(p, &e);                  // |m| in [0.5, 1)
+  const double r = std::nearbyint(std::ldexp(m, 8));    // |r| in [128, 256], integer, ties to even
+  const float f = static_cast<float>(std::ldexp(r, e - 8));  // exact: r has at most 9 bits
+  uint32_t u;
+  std::memcpy(&u, &f, sizeof u);
+  return static_cast<uint16_t>(u >> 16);
+}
+
+// stored[b][i][j] = bf16(Delta[128 b + i] * blocks[b][i][j]); smooth == nullptr means Delta = 1.
+void oracle_dense_stored_blocks(const float* blocks, const float* smooth, int K, uint16_t* stored) {
+  const int nb = K / kBlock;
+  for (int b = 0; b < nb; ++b)
+    for (int i = 0; i < kBlock; ++i) {
+      const double delta = smooth ? static_cast<double>(smooth[b * kBlock + i]) : 1.0;
+      for (int j = 0; j < kBlock; ++j) {
+        const int64_t at = (static_cast<int64_t>(b) * kBlock + i) * kBlock + j;
+        stored[at] = double_to_bf16_bits(delta * static_cast<double>(blocks[at]));  // product of two floats: exact in double
+      }
+    }
+}
+
+// v[m, 128 b + j] = fl32( sum_i x[m, 128 b + i] * S_b[i][j] ), the sum taken in double in index order
+// (every product of two bf16 values is exact).
+void oracle_rotate_dense(const uint16_t* x_bf16, int64_t ldx, int M, int K, const uint16_t* stored, float* v) {
+  const int nb = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int b = 0; b < nb; ++b)
+      for (int j = 0; j < kBlock; ++j) {
+        double s = 0.0;
+        for (int i = 0; i < kBlock; ++i)
+          s += static_cast<double>(bf16_to_float(x_bf16[m * ldx + b * kBlock + i])) *
+               static_cast<double>(bf16_to_float(stored[(static_cast<int64_t>(b) * kBlock + i) * kBlock + j]));
+        v[static_cast<int64_t>(m) * K + b * kBlock + j] = static_cast<float>(s);
+      }
+}
+
+// inv[b] = S_b^-1 in double: Gauss-Jordan elimination with partial pivoting on [S | I].
+// Returns 0, or 1 + the index of the first singular block.
+int oracle_invert_blocks(const uint16_t* stored, int nb, double* inv) {
+  const int n = kBlock;
+  for (int b = 0; b < nb; ++b) {
+    std::vector<double> a(static_cast<size_t>(n) * n);
+    double* x = inv + static_cast<int64_t>(b) * n * n;
+    for (int i = 0; i < n; ++i)
+      for (int j = 0; j < n; ++j) {
+        a[i * n + j] = static_cast<double>(bf16_to_float(stored[(static_cast<int64_t>(b) * n + i) * n + j]));
+        x[i * n + j] = i == j ? 1.0 : 0.0;
+      }
+    for (int c = 0; c < n; ++c) {
+      int piv = c;
+      for (int r = c + 1; r < n; ++r)
+        if (std::fabs(a[r * n + c]) > std::fabs(a[piv * n + c])) piv = r;
+      if (a[piv * n + c] == 0.0) return b + 1;
+      if (piv != c)
+        for (int j = 0; j < n; ++j) {
+          std::swap(a[c * n + j], a[piv * n + j]);
+          std::swap(x[c * n + j], x[piv * n + j]);
+        }
+      const double d = a[c * n + c];
+      for (int j = 0; j < n; ++j) {
+        a[c * n + j] /= d;
+        x[c * n + j] /= d;
+      }
+      for (int r = 0; r < n; ++r) {
+        if (r == c) continue;
+        const double f = a[r * n + c];
+        if (f == 0.0) continue;
+        for (int j = 0; j < n; ++j) {
+          a[r * n + j] -= f * a[c * n + j];
+          x[r * n + j] -= f * x[c * n + j];
+        }
+      }
+    }
+  }
+  return 0;
+}
+
+// Weight side of Eq. 10 with dense blocks: wr[n, 128 b + j] = fl32( sum_i inv_b[j][i] * W[n, 128 b + i] ),
+// i.e. the column vector S_b^-1 w; products and sums in double, in index order, each rounded separately.
+void oracle_prepare_dense_rotate(const uint16_t* w_bf16, int N, int K, const double* inv, float* wr) {
+  const int nb = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int b = 0; b < nb; ++b)
+      for (int j = 0; j < kBlock; ++j) {
+        double s = 0.0;
+        for (int i = 0; i < kBlock; ++i)
+          s += inv[(static_cast<int64_t>(b) * kBlock + j) * kBlock + i] *
+               static_cast<double>(bf16_to_float(w_bf16[static_cast<int64_t>(n) * K + b * kBlock + i]));
+        wr[static_cast<int64_t>(n) * K + b * kBlock + j] = static_cast<float>(s);
+      }
+}
+
+// 4-bit quantiser on already-rotated fp32 weight rows (same format as oracle_prepare_w4).
+void oracle_quantize_w4_rows(const float* wr, int N, int K, uint8_t* packed, float* scales) {
+  const int groups = K / kBlock;
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int kg = 0; kg < groups; ++kg) {
+      int8_t q[kBlock];
+      scales[static_cast<int64_t>(n) * groups + kg] = quantize_span(wr + static_cast<int64_t>(n) * K + kg * kBlock, kBlock, 7.0f, q);
+      for (int i = 0; i < kBlock; i += 2) {
+        const uint8_t lo = static_cast<uint8_t>(q[i]) & 0xF;
+        const uint8_t hi = static_cast<uint8_t>(q[i + 1]) & 0xF;
+        packed[(static_cast<int64_t>(n) * K + kg * kBlock + i) / 2] = static_cast<uint8_t>(lo | (hi << 4));
+      }
+    }
+}
+
+// ---- greedy construction of one block (Sec. 3.2, Eq. 6-7) ------------------------------------------------
+// Eq. 6: R^k = C1 Q C2.  C1 swaps the first column with the column holding the largest-magnitude entry of the
+// current activations; Q is a random orthogonal matrix whose first row is uniform (every entry 1/sqrt(128)),
+// so the outlier now sitting in position 0 is spread evenly over all outputs; C2 swaps the two columns back.
+// The random part of Q is an input: a Gaussian draw G per step.  Row 0 of Q is the uniform row, rows 1..127
+// are G's rows 1..127 made orthonormal to all earlier rows by modified Gram-Schmidt.
+static void uniform_first_row_orthogonal(const double* G, double* Q) {
+  const int n = kBlock;
+  for (int j = 0; j < n; ++j) Q[j] = 1.0 / std::sqrt(static_cast<double>(n));
+  for (int r = 1; r < n; ++r) {
+    double* q = Q + r * n;
+    for (int j = 0; j < n; ++j) q[j] = G[r * n + j];
+    for (int s = 0; s < r; ++s) {
+      double dot = 0.0;
+      for (int j = 0; j < n; ++j) dot += q[j] * Q[s * n + j];
+      for (int j = 0; j < n; ++j) q[j] -= dot * Q[s * n + j];
+    }
+    double nrm = 0.0;
+    for (int j = 0; j < n; ++j) nrm += q[j] * q[j];
+    nrm = std::sqrt(nrm);
+    for (int j = 0; j < n; ++j) q[j] /= nrm;
+  }
+}
+
+// Eq. 7: R = R^1 R^2 ... R^n with n = argmin_k max_ij |(X R^1 ... R^k)_ij| over k = 1..steps (the first k
+// reaching the minimum).  Xc: calibration activations of this block [Mc, 128]; gauss: [steps][128][128].
+// Outputs the product R [128][128], the per-step maxima trace[steps], and returns n.
+int oracle_greedy_block(const double* Xc, int Mc, int steps, const double* gauss, double* R, double* trace) {
+  const int n = kBlock;
+  std::vector<double> Y(Xc, Xc + static_cast<size_t>(Mc) * n), Yn(static_cast<size_t>(Mc) * n);
+  std::vector<double> P(static_cast<size_t>(n) * n, 0.0), Pn(static_cast<size_t>(n) * n), Q(static_cast<size_t>(n) * n), Rk(static_cast<size_t>(n) * n);
+  for (int i = 0; i < n; ++i) P[i * n + i] = 1.0;
+  int best_k = 0;
+  double best = 0.0;
+  for (int k = 1; k <= steps; ++k) {
+    int d = 0;
+    double mx = -1.0;
+    for (int m = 0; m < Mc; ++m)
+      for (int j = 0; j < n; ++j)
+        if (std::fabs(Y[static_cast<size_t>(m) * n + j]) > mx) {
+          mx = std::fabs(Y[static_cast<size_t>(m) * n + j]);
+          d = j;
+        }
+    uniform_first_row_orthogonal(gauss + static_cast<size_t>(k - 1) * n * n, Q.data());
+    // (C1 Q C2)[i][j] = Q[s(i)][s(j)] with s the transposition of 0 and d
+    for (int i = 0; i < n; ++i) {
+      const int si = i == 0 ? d : (i == d ? 0 : i);
+      for (int j = 0; j < n; ++j) {
+        const int sj = j == 0 ? d : (j == d ? 0 : j);
+        Rk[i * n + j] = Q[si * n + sj];
+      }
+    }
+    for (int m = 0; m < Mc; ++m)
+      for (int j = 0; j < n; ++j) {
+        double s = 0.0;
+        for (int i = 0; i < n; ++i) s += Y[static_cast<size_t>(m) * n + i] * Rk[i * n + j];
+        Yn[static_cast<size_t>(m) * n + j] = s;
+      }
+    Y.swap(Yn);
+    for (int a = 0; a < n; ++a)
+      for (int j = 0; j < n; ++j) {
+        double s = 0.0;
+        for (int i = 0; i < n; ++i) s += P[a * n + i] * Rk[i * n + j];
+        Pn[a * n + j] = s;
+      }
+    P.swap(Pn);
+    double now = 0.0;
+    for (size_t i = 0; i < Y.size(); ++i) now = std::fmax(now, std::fabs(Y[i]));
+    trace[k - 1] = now;
+    if (best_k == 0 || now < best) {
+      best = now;
+      best_k = k;
+      std::memcpy(R, P.data(), sizeof(double) * n * n);
+    }
+  }
+  return best_k;
+}
+
 int oracle_num_threads() {
   int n = 1;
 #ifdef _OPENMP

@@ -23,6 +23,8 @@ def _lib() -> C.CDLL:
         _LIB = C.CDLL(_build.build())
         _LIB.oracle_group_of.restype = C.c_int
         _LIB.oracle_num_threads.restype = C.c_int
+        _LIB.oracle_invert_blocks.restype = C.c_int
+        _LIB.oracle_greedy_block.restype = C.c_int
     return _LIB
 
 
@@ -253,3 +255,60 @@ def linear_asym_rows(q, sx, zp, qw, sw, bias_bits, rows) -> np.ndarray:
     _lib().oracle_linear_asym_rows(_p(q), _p(_c(sx, np.float32)), _p(_c(zp, np.int32)), _p(qw), _p(_c(sw, np.float32)), _p(b),
                                    _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), _p(y))
     return y
+
+
+# ---- dense block rotations (Eq. 6-8) -------------------------------------------------------------
+
+def dense_stored_blocks(blocks, smooth_g=None) -> np.ndarray:
+    """bf16 bit patterns [K/128, 128, 128] of Delta-scaled blocks, as applied to the activations."""
+    b = _c(blocks, np.float32)
+    nb = b.shape[0]
+    sm = None if smooth_g is None else _c(smooth_g, np.float32)
+    out = np.empty((nb, 128, 128), np.uint16)
+    _lib().oracle_dense_stored_blocks(_p(b), _p(sm), C.c_int(nb * 128), _p(out))
+    return out
+
+
+def rotate_dense(x_bits, stored) -> np.ndarray:
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    v = np.empty((M, K), np.float32)
+    _lib().oracle_rotate_dense(_p(x), C.c_int64(K), C.c_int(M), C.c_int(K), _p(_c(stored, np.uint16)), _p(v))
+    return v
+
+
+def invert_blocks(stored) -> np.ndarray:
+    s = _c(stored, np.uint16)
+    inv = np.empty(s.shape, np.float64)
+    rc = int(_lib().oracle_invert_blocks(_p(s), C.c_int(s.shape[0]), _p(inv)))
+    if rc != 0:
+        raise ValueError(f"block {rc - 1} is singular")
+    return inv
+
+
+def prepare_dense_rotate(w_bits, inv) -> np.ndarray:
+    w = _c(w_bits, np.uint16)
+    N, K = w.shape
+    wr = np.empty((N, K), np.float32)
+    _lib().oracle_prepare_dense_rotate(_p(w), C.c_int(N), C.c_int(K), _p(_c(inv, np.float64)), _p(wr))
+    return wr
+
+
+def quantize_w4_rows(wr) -> Tuple[np.ndarray, np.ndarray]:
+    wr = _c(wr, np.float32)
+    N, K = wr.shape
+    packed = np.empty((N, K // 2), np.uint8)
+    scales = np.empty((N, K // 128), np.float32)
+    _lib().oracle_quantize_w4_rows(_p(wr), C.c_int(N), C.c_int(K), _p(packed), _p(scales))
+    return packed, scales
+
+
+def greedy_block(x_calib, gauss) -> Tuple[np.ndarray, int, np.ndarray]:
+    """(R [128,128] fp64, n, per-step maxima) of Eq. 6-7 for one block."""
+    x = _c(x_calib, np.float64)
+    g = _c(gauss, np.float64)
+    steps = g.shape[0]
+    R = np.empty((128, 128), np.float64)
+    trace = np.empty(steps, np.float64)
+    n = int(_lib().oracle_greedy_block(_p(x), C.c_int(x.shape[0]), C.c_int(steps), _p(g), _p(R), _p(trace)))
+    return R, n, trace

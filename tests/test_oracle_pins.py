@@ -556,3 +556,159 @@ def test_asymmetric_linear_brute_force_and_accuracy():
     err_a = np.linalg.norm(sa[:, None] * (qa.astype(np.float64) - za[:, None]) - v)
     err_s = np.linalg.norm(ss[:, None] * qs.astype(np.float64) - v)
     assert err_a < 0.6 * err_s
+
+
+# --------------------------------------------------------------------------- #
+# dense block rotations (Eq. 6-8)
+# --------------------------------------------------------------------------- #
+def _random_orthogonal_blocks(nb, seed):
+    rng = np.random.default_rng(seed)
+    out = np.empty((nb, 128, 128), np.float32)
+    for b in range(nb):
+        q, r = np.linalg.qr(rng.standard_normal((128, 128)))
+        out[b] = (q * np.sign(np.diag(r))).astype(np.float32)
+    return out
+
+
+def _sylvester(n):
+    H = np.ones((1, 1))
+    while H.shape[0] < n:
+        H = np.block([[H, H], [H, -H]])
+    return H
+
+
+def test_dense_blocks_are_stored_as_nearest_bf16():
+    rng = np.random.default_rng(40)
+    blocks = _random_orthogonal_blocks(2, 41)
+    smooth = rng.uniform(0.1, 8.0, 256).astype(np.float32)
+    stored = f32_of(O.dense_stored_blocks(blocks, smooth)).astype(np.float64)
+    exact = blocks.astype(np.float64) * smooth.astype(np.float64).reshape(2, 128, 1)  # row i of block b scaled by Delta[128 b + i]
+    # nearest bf16: the error is at most half a unit of the last of the 8 significand bits
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(stored))) - 7)
+    assert np.all(np.abs(stored - exact) <= ulp / 2)
+    assert np.max(np.abs(stored - exact) / ulp) > 0.49            # and the bound is attained: it is not a finer format
+    assert np.array_equal(bf16(stored), O.dense_stored_blocks(blocks, smooth))   # the stored values are bf16 numbers
+    # without smoothing the blocks themselves are rounded
+    assert np.array_equal(O.dense_stored_blocks(blocks, None), bf16(blocks))
+    # ties go to even: 1 + 2^-8 lies midway between 1 and 1 + 2^-7 -> 1; 1 + 3 * 2^-8 -> 1 + 2^-6
+    tie = np.zeros((1, 128, 128), np.float32)
+    tie[0, 0, 0] = 1.0 + 2.0 ** -8
+    tie[0, 0, 1] = 1.0 + 3 * 2.0 ** -8
+    tie[0, 1, 0] = 3.0                      # times Delta = 1/3 rounded to fp32: product needs the double
+    sm = np.ones(128, np.float32)
+    got = f32_of(O.dense_stored_blocks(tie, sm))
+    assert got[0, 0, 0] == 1.0 and got[0, 0, 1] == np.float32(1.0 + 2.0 ** -6)
+
+
+def test_dense_rotation_is_the_matrix_product():
+    rng = np.random.default_rng(42)
+    K, M = 384, 24
+    blocks = _random_orthogonal_blocks(K // 128, 43)
+    smooth = rng.uniform(0.2, 5.0, K).astype(np.float32)
+    stored_bits = O.dense_stored_blocks(blocks, smooth)
+    S = f32_of(stored_bits).astype(np.float64)
+    x_bits = bf16(rng.standard_normal((M, K)) * 3.0)
+    x = f32_of(x_bits).astype(np.float64)
+    v = O.rotate_dense(x_bits, stored_bits).astype(np.float64)
+    ref = np.concatenate([x[:, 128 * b:128 * (b + 1)] @ S[b] for b in range(K // 128)], axis=1)  # BLAS, another summation order
+    bound = np.concatenate([np.abs(x[:, 128 * b:128 * (b + 1)]) @ np.abs(S[b]) for b in range(K // 128)], axis=1)
+    assert np.all(np.abs(v - ref) <= bound * 2.0 ** -23)       # one fp32 rounding of an (almost) exact sum
+    # a transposed operand would fail this by O(1)
+    wrong = np.concatenate([x[:, 128 * b:128 * (b + 1)] @ S[b].T for b in range(K // 128)], axis=1)
+    assert np.max(np.abs(v - wrong)) > 0.5
+
+
+def test_dense_rotation_with_hadamard_block_equals_the_butterfly():
+    # S = H_128 / 8 is bf16-exact; with small integer rows both evaluations are exact, so the dense product must
+    # equal the butterfly of the single-rotation path bit for bit (two structurally different routes).
+    rng = np.random.default_rng(44)
+    H = _sylvester(128)
+    blocks = np.stack([H / 8.0, -H / 8.0]).astype(np.float32)
+    stored = O.dense_stored_blocks(blocks, None)
+    x_bits = bf16(rng.integers(-9, 10, (16, 256)).astype(np.float64))
+    vec = np.concatenate([np.full(128, 0.125, np.float32), np.full(128, -0.125, np.float32)])
+    assert np.array_equal(O.rotate_dense(x_bits, stored), O.rotate(x_bits, vec))
+
+
+def test_dense_block_inverse_and_invariance_fp64():
+    rng = np.random.default_rng(45)
+    K, M, N = 256, 12, 20
+    blocks = _random_orthogonal_blocks(K // 128, 46)
+    smooth = rng.uniform(0.05, 20.0, K).astype(np.float32)
+    stored_bits = O.dense_stored_blocks(blocks, smooth)
+    S = f32_of(stored_bits).astype(np.float64)
+    inv = O.invert_blocks(stored_bits)
+    for b in range(K // 128):
+        assert np.max(np.abs(S[b] @ inv[b] - np.eye(128))) < 1e-10
+        assert np.max(np.abs(inv[b] - np.linalg.inv(S[b]))) < 1e-9 * np.max(np.abs(inv[b]))   # LAPACK's LU, not Gauss-Jordan
+    # Eq. 9 / Eq. 10: (X S)(S^-1 W^T) = X W^T
+    x_bits = bf16(rng.standard_normal((M, K)))
+    w_bits = bf16(rng.standard_normal((N, K)) * 0.05)
+    x = f32_of(x_bits).astype(np.float64)
+    w = f32_of(w_bits).astype(np.float64)
+    xs = np.concatenate([x[:, 128 * b:128 * (b + 1)] @ S[b] for b in range(K // 128)], axis=1)
+    wr = O.prepare_dense_rotate(w_bits, inv).astype(np.float64)
+    wr_ref = np.concatenate([w[:, 128 * b:128 * (b + 1)] @ np.linalg.inv(S[b]).T for b in range(K // 128)], axis=1)
+    assert np.max(np.abs(wr - wr_ref)) <= 2.0 ** -22 * np.max(np.abs(wr_ref))
+    y = xs @ wr.T
+    y_ref = x @ w.T
+    assert np.max(np.abs(y - y_ref)) <= 1e-5 * np.max(np.abs(y_ref))   # wr is rounded to fp32: 2^-24 per term
+    # a singular block is reported
+    bad = stored_bits.copy()
+    bad[1, :, 5] = bad[1, :, 7]
+    with pytest.raises(ValueError):
+        O.invert_blocks(bad)
+
+
+def test_quantize_w4_rows_matches_the_hadamard_path_format():
+    # the stand-alone 4-bit quantiser must produce what prepare_w4 produces from the same rotated rows
+    rng = np.random.default_rng(47)
+    N, K = 16, 256
+    signs = (rng.integers(0, 2, K) * 2 - 1).astype(np.int8)
+    _, wv = O.fused_vectors(signs, None)
+    w_bits = bf16(rng.standard_normal((N, K)) * 0.02)
+    packed_ref, scales_ref = O.prepare_w4(w_bits, wv)
+    packed, scales = O.quantize_w4_rows(O.rotate(w_bits, wv))
+    assert np.array_equal(packed, packed_ref) and np.array_equal(scales, scales_ref)
+
+
+def test_greedy_block_single_outlier_closed_form():
+    # one massive column d, everything else zero: C1 moves it to position 0, the uniform first row of Q spreads
+    # it as a / sqrt(128) over all outputs, C2 swaps two equal entries -> every entry equals a / sqrt(128).
+    rng = np.random.default_rng(48)
+    Mc, d = 6, 37
+    a = rng.uniform(20.0, 50.0, Mc) * np.where(rng.random(Mc) < 0.5, -1.0, 1.0)
+    X = np.zeros((Mc, 128))
+    X[:, d] = a
+    R, n, trace = O.greedy_block(X, rng.standard_normal((1, 128, 128)))
+    assert n == 1
+    assert np.max(np.abs(R @ R.T - np.eye(128))) < 1e-12
+    Y = X @ R
+    assert np.allclose(Y, np.repeat((a / np.sqrt(128.0))[:, None], 128, axis=1), rtol=0, atol=1e-12)
+    assert np.isclose(trace[0], np.max(np.abs(a)) / np.sqrt(128.0))
+
+
+def test_greedy_block_eq6_structure_and_eq7_choice():
+    rng = np.random.default_rng(49)
+    Mc, steps = 64, 6
+    X = rng.standard_normal((Mc, 128))
+    X[:, 11] *= 60.0
+    X[:, 90] *= 25.0
+    G = rng.standard_normal((steps, 128, 128))
+    R, n, trace = O.greedy_block(X, G)
+    assert np.max(np.abs(R @ R.T - np.eye(128))) < 1e-11            # product of orthogonal factors
+    assert 1 <= n <= steps and n == int(np.argmin(trace)) + 1        # Eq. 7: the first k reaching the minimum
+    assert np.isclose(np.max(np.abs(X @ R)), trace[n - 1], rtol=1e-12)
+    assert trace[n - 1] < 0.25 * np.max(np.abs(X))                   # the massive outliers are gone
+    # rebuild the first factor from Eq. 6 with numpy: Q by QR of [uniform row; G rows] (Gram-Schmidt up to row signs)
+    d = int(np.argmax(np.max(np.abs(X), axis=0)))
+    assert d == 11
+    A = G[0].copy()
+    A[0] = 1.0 / np.sqrt(128.0)
+    q, r = np.linalg.qr(A.T)
+    Q = (q * np.sign(np.diag(r))).T                                   # rows orthonormal, row 0 = +uniform
+    C = np.eye(128)
+    C[[0, d]] = C[[d, 0]]
+    R1 = C @ Q @ C
+    R_one, n_one, _ = O.greedy_block(X, G[:1])
+    assert n_one == 1 and np.max(np.abs(R_one - R1)) < 1e-10
