@@ -212,6 +212,44 @@ trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const
 trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
                              int32_t M, const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
 
+/* Dense block rotations (Sec. 3.2, Eq. 6-8): R = BlockDiag(R_b1 .. R_bK) with dense 128 x 128 orthogonal blocks, one
+ * set per time-step group (Eq. 10).  blocks: host fp32 [G][K/128][128][128], R_b[i][j] with i the input channel
+ * (v = x R).  smooth: host [G][K] (> 0) or NULL, the multiplier Delta_t of Eq. 10, folded into the rows of each block.
+ * The scaled blocks are STORED IN BF16, S_b[i][j] = bf16(Delta[128 b + i] * R_b[i][j]) (nearest, ties to even), because
+ * that is the format the tensor cores apply them in; the weight side (trdq_prepare_weights with this object, 8- or 4-bit)
+ * multiplies by the exact inverse of the stored S_b, computed on the host in double, so the product
+ * G_t(X) . H_t(W) = X W of Eq. 9 is preserved whatever the rounding did:
+ *   wr[n, 128 b + j] = fl32( sum_i (S_b^-1)[j][i] * W[n, 128 b + i] )      sums in double, i ascending.
+ * TRDQ_ERR_GROUP: bounds not ascending, a non-positive smooth value, a non-finite product or a singular block.
+ * The object is accepted by trdq_prepare_weights, trdq_group_of, trdq_rotate_dense_quantize and
+ * trdq_rotation_destroy; the Hadamard entry points (trdq_rotate_quantize, _asym, trdq_run_layers) return TRDQ_ERR_MISMATCH. */
+trdq_status trdq_rotation_create_dense(int32_t K, int32_t num_groups, const int32_t* t_bounds, const float* blocks, const float* smooth,
+                                       trdq_rotation** out);
+
+/* Online side with dense blocks: v[m, 128 b + j] = sum_i X[m, 128 b + i] * S_b[i][j] on the tensor cores (bf16 operands, every
+ * product exact, fp32 accumulation), then the per-token quantizer of trdq_rotate_quantize on v (same scale and code
+ * definitions).  The row maximum must be known before the first code, so X is read twice; `workspace` (device,
+ * 4-byte aligned, at least the size trdq_rotate_dense_workspace reports = 4 * (K/128) * M bytes) holds the per-block row
+ * maxima between the two passes.  It is scratch: no initialisation needed, contents undefined afterwards; two calls that
+ * may overlap on the GPU need separate workspaces.  Asynchronous on `stream`; allocates nothing.
+ * TRDQ_ERR_MISMATCH if rot was not made by trdq_rotation_create_dense; TRDQ_ERR_NOMEM if the workspace is too small;
+ * otherwise the errors of trdq_rotate_quantize.  Because the accumulation order inside the tensor cores is not
+ * specified, v agrees with the exactly rounded sum only to a few units of 2^-24 * sum_i |x_i S_ij|; codes can differ by
+ * one step from an exactly rounded evaluation where v * 127 / amax falls that close to a rounding boundary. */
+trdq_status trdq_rotate_dense_workspace(const trdq_rotation* rot, int32_t M, uint64_t* bytes);
+trdq_status trdq_rotate_dense_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, int8_t* codes,
+                                       float* scales, void* workspace, uint64_t workspace_bytes, void* stream);
+
+/* Greedy construction of ONE block (Eq. 6-7), on the host in double; offline calibration, no GPU work.
+ * x_calib: host fp32 [rows][128], calibration activations of the block's 128 channels.  gauss: host double
+ * [steps][128][128], the random draws of the method (standard normal), passed in so that the result is reproducible.
+ * Step k: C swaps column 0 with the column holding the largest |entry| of the current activations; Q_k has the uniform
+ * first row 1/sqrt(128) and rows 1..127 from gauss[k-1] made orthonormal by Gram-Schmidt; R^k = C Q_k C (Eq. 6).  The
+ * result is R^1 R^2 .. R^n with n the first step that minimises max |X R^1 .. R^n| (Eq. 7), written to R_out [128][128]
+ * (fp32) and *n_used (may be NULL).  TRDQ_ERR_GROUP for non-finite inputs or a degenerate draw. */
+trdq_status trdq_greedy_rotation_block(const float* x_calib, int32_t rows, int32_t steps, const double* gauss, float* R_out,
+                                       int32_t* n_used);
+
 /* One quantized linear layer of a denoising step: rotate + quantize X into the caller's code and
  * scale buffers, then the integer GEMM with its epilogue into Y (shapes as in the two calls above). */
 typedef struct trdq_layer_op {

@@ -242,6 +242,8 @@ trdq_status trdq_rotation_destroy(trdq_rotation* rot) {
   if (rot->weight_vec) cudaFree(rot->weight_vec);
   if (rot->perm) cudaFree(rot->perm);
   if (rot->vec2) cudaFree(rot->vec2);
+  if (rot->dense) cudaFree(rot->dense);
+  if (rot->dense_inv_t) cudaFree(rot->dense_inv_t);
   delete rot;
   return TRDQ_OK;
 }
@@ -298,7 +300,26 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
       trdq_weights_destroy(w);
       return TRDQ_ERR_NOMEM;
     }
+    if (rot->dense) {
+      // dense blocks (Eq. 6-8): W S^-1 into an fp32 scratch, then the quantizer
+      float* wr = nullptr;
+      if (cudaMalloc(&wr, static_cast<size_t>(N) * K * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_NOMEM;
+      }
+      const size_t per_group = static_cast<size_t>(K / TRDQ_BLOCK) * TRDQ_BLOCK * TRDQ_BLOCK;
+      const cudaError_t ed = launch_dense_prepare(W_bf16, N, K, rot->dense_inv_t + static_cast<size_t>(g) * per_group, wbits, wr, gw.codes,
+                                                  gw.scales, static_cast<cudaStream_t>(stream));
+      const cudaError_t es = ed == cudaSuccess ? cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) : ed;  // the scratch is freed next
+      cudaFree(wr);
+      if (es != cudaSuccess) {
+        trdq_weights_destroy(w);
+        return TRDQ_ERR_CUDA;
+      }
+    }
     const cudaError_t e =
+        rot->dense ? cudaSuccess :
         rot->perm ? launch_rotate2_quantize(W_bf16, K, N, K, rot->weight_vec + static_cast<size_t>(g) * K, rot->perm + static_cast<size_t>(g) * K,
                                             rot->vec2 + static_cast<size_t>(g) * K, wbits == 8 ? 0 : 1, gw.codes, gw.scales,
                                             static_cast<cudaStream_t>(stream))
@@ -398,6 +419,7 @@ trdq_status trdq_weights_export(const trdq_weights* w, int32_t g, void* codes_ou
 trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, int8_t* codes,
                                  float* scales, void* stream) {
   if (!rot) return TRDQ_ERR_NULL;
+  if (rot->dense) return TRDQ_ERR_MISMATCH;  // dense blocks need the workspace of trdq_rotate_dense_quantize
   if (M < 0) return TRDQ_ERR_SHAPE;
   const int g = find_group(rot->t_bounds, t);
   if (g < 0) return TRDQ_ERR_TIMESTEP;
@@ -500,6 +522,7 @@ trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const in
 trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, uint8_t* codes,
                                       float* scales, int32_t* zero_points, void* stream) {
   if (!rot) return TRDQ_ERR_NULL;
+  if (rot->dense) return TRDQ_ERR_MISMATCH;
   if (M < 0 || rot->K > 10240 || rot->perm) return TRDQ_ERR_SHAPE;
   const int g = find_group(rot->t_bounds, t);
   if (g < 0) return TRDQ_ERR_TIMESTEP;
@@ -545,7 +568,7 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
   for (int i = 0; i < count; ++i) {
     const trdq_layer_op& op = ops[i];
     if (!op.rot || !op.w) return TRDQ_ERR_NULL;
-    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds) return TRDQ_ERR_MISMATCH;
+    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds || op.rot->dense) return TRDQ_ERR_MISMATCH;
     if (find_group(op.rot->t_bounds, t) < 0) return TRDQ_ERR_TIMESTEP;
     if (op.M < 0 || op.ldx < op.rot->K || op.ldy < op.w->N) return TRDQ_ERR_SHAPE;
     if (op.M > 0 && (!op.X_bf16 || !op.codes || !op.scales || !op.Y_bf16)) return TRDQ_ERR_NULL;

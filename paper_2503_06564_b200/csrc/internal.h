@@ -18,6 +18,10 @@ struct trdq_rotation {
   // full balancing transform (Eq. 9) only; perm == nullptr means the single-rotation path
   int32_t* perm = nullptr;        // dev [G][K]: (v P)[j] = v[perm[j]]
   float* vec2 = nullptr;          // dev [G][K]: d2 * 2^-3.5, scaling before the second rotation
+  // dense block rotations (Eq. 6-8) only; dense == nullptr means a Hadamard path
+  uint16_t* dense = nullptr;      // dev bf16 [G][K/128][128 j][128 i]: S_b[i][j] = bf16(Delta_i R_b[i][j]), stored transposed
+  double* dense_inv_t = nullptr;  // dev [G][K/128][128 i][128 j] = (S_b^-1)[j][i], for the weight side
+  CUtensorMap tmap_dense;         // `dense` as a [G * K/128 * 128, 128] bf16 matrix, box 64 x 128, 128-byte swizzle
 };
 
 namespace trdq {
@@ -64,6 +68,14 @@ int rotate_quantize_tma_rows(int32_t K);  // rows per tile, 0 if K is too wide f
 bool rotate_quantize_prefers_tma(int32_t M, int32_t K);
 trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
                                        float* scales, cudaStream_t stream);
+
+// rotate_dense.cu: dense block rotation on the tensor cores + per-token quantizer (two passes over X)
+uint64_t rotate_dense_workspace_bytes(int32_t M, int32_t K);
+trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const void* x_bf16, int64_t ldx, int32_t M, int8_t* codes,
+                                         float* scales, float* workspace, cudaStream_t stream);
+// weight side: wr = W S^-1 (fp64 sums, one fp32 rounding) into wr_scratch [N,K], then the 8- or 4-bit quantizer
+cudaError_t launch_dense_prepare(const void* w_bf16, int32_t N, int32_t K, const double* inv_t, int wbits, float* wr_scratch,
+                                 void* codes, float* scales, cudaStream_t stream);
 
 // gemm_i8.cu
 struct GemmSegment {

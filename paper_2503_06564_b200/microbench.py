@@ -2,6 +2,7 @@
 
     python -m paper_2503_06564_b200.microbench rq   --M 65536 --K 1152
     python -m paper_2503_06564_b200.microbench gemm --M 16384 --K 1152 --N 4608
+    python -m paper_2503_06564_b200.microbench rqd  --M 16384 --K 1152      (dense block rotation, Eq. 6-8)
 
 Also the small, self-ending command to put under a profiler (few launches, a few hundred MB).
 Buffers are rotated through `--sets` distinct copies so that consecutive launches do not find
@@ -19,7 +20,7 @@ def main():
     import torch
     from paper_2503_06564_b200 import build, trdq
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["rq", "gemm"])
+    ap.add_argument("kernel", choices=["rq", "rqd", "gemm"])
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--K", type=int, default=1152)
     ap.add_argument("--N", type=int, default=4608)
@@ -41,7 +42,19 @@ def main():
     xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(args.sets)]
     codes = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(args.sets)]
     scales = [torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(args.sets)]
-    if args.kernel == "rq":
+    if args.kernel == "rqd":
+        blocks = np.empty((1, K // 128, 128, 128), np.float32)
+        for b in range(K // 128):
+            q, _ = np.linalg.qr(rng.standard_normal((128, 128)))
+            blocks[0, b] = q
+        drot = trdq.DenseRotation(K, [0, 1000], blocks, None)
+        ws = torch.empty((trdq.trdq_rotate_dense_workspace(drot, M),), dtype=torch.uint8, device="cuda")
+
+        def run(i):
+            s = i % args.sets
+            trdq.trdq_rotate_dense_quantize(drot, 0, xs[s], codes[s], scales[s], ws)
+        work, unit = M * (3.0 * K + 4.0) / 1e9, "GB/s"
+    elif args.kernel == "rq":
         def run(i):
             s = i % args.sets
             trdq.trdq_rotate_quantize(rot, 0, xs[s], codes[s], scales[s])

@@ -29,7 +29,8 @@ EXPORTS = (
     "trdq_rotate_quantize", "trdq_linear", "trdq_linear_cfg", "trdq_gemm_i32", "trdq_device_status",
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
     "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
-    "trdq_selftest_wait_expiry",
+    "trdq_selftest_wait_expiry", "trdq_rotation_create_dense", "trdq_rotate_dense_workspace", "trdq_rotate_dense_quantize",
+    "trdq_greedy_rotation_block",
 )
 
 
@@ -87,6 +88,11 @@ def lib() -> C.CDLL:
         l.trdq_rotate_quantize_asym.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp]
         l.trdq_linear_asym.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_selftest_wait_expiry.argtypes = [vp]
+        l.trdq_rotation_create_dense.argtypes = [i32, i32, C.POINTER(i32), C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(vp)]
+        l.trdq_rotate_dense_workspace.argtypes = [vp, i32, C.POINTER(C.c_uint64)]
+        l.trdq_rotate_dense_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, C.c_uint64, vp]
+        l.trdq_greedy_rotation_block.argtypes = [C.POINTER(C.c_float), i32, i32, C.POINTER(C.c_double), C.POINTER(C.c_float),
+                                                 C.POINTER(i32)]
         l.trdq_device_status.argtypes = [C.POINTER(C.c_uint32)]
         _lib = l
     return _lib
@@ -167,6 +173,24 @@ class Rotation:
             pass
 
 
+class DenseRotation(Rotation):
+    """Handle of a trdq_rotation made of dense 128 x 128 blocks (Eq. 6-8): blocks fp32 [G][K/128][128][128]."""
+
+    def __init__(self, K: int, t_bounds, blocks, smooth=None):
+        self._h = C.c_void_p()
+        b = np.ascontiguousarray(t_bounds, dtype=np.int32)
+        G = int(len(b) - 1)
+        blk = np.ascontiguousarray(blocks, dtype=np.float32)
+        assert blk.shape == (G, int(K) // 128, 128, 128), blk.shape
+        sm = None if smooth is None else np.ascontiguousarray(smooth, dtype=np.float32)
+        _check(lib().trdq_rotation_create_dense(int(K), G, b.ctypes.data_as(C.POINTER(C.c_int32)),
+                                                blk.ctypes.data_as(C.POINTER(C.c_float)),
+                                                None if sm is None else sm.ctypes.data_as(C.POINTER(C.c_float)),
+                                                C.byref(self._h)), "trdq_rotation_create_dense")
+        self.K = int(K)
+        self.num_groups = G
+
+
 class Weights:
     """Handle of a trdq_weights (H_t(W) of one layer, quantized for every group)."""
 
@@ -229,6 +253,43 @@ def trdq_rotate_quantize(rot: Rotation, t: int, X_bf16, codes=None, scales=None)
     _check(lib().trdq_rotate_quantize(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(codes), _ptr(scales), _stream()),
            "trdq_rotate_quantize")
     return codes, scales
+
+
+def trdq_rotate_dense_workspace(rot: Rotation, M: int) -> int:
+    n = C.c_uint64(0)
+    _check(lib().trdq_rotate_dense_workspace(rot._h, int(M), C.byref(n)), "trdq_rotate_dense_workspace")
+    return int(n.value)
+
+
+def trdq_rotate_dense_quantize(rot: Rotation, t: int, X_bf16, codes=None, scales=None, workspace=None):
+    """codes int8 [M,K], scales fp32 [M] of the activations rotated by the dense blocks of time-step t."""
+    import torch
+    assert X_bf16.is_cuda and X_bf16.dim() == 2 and X_bf16.element_size() == 2 and X_bf16.stride(1) == 1
+    M = int(X_bf16.shape[0])
+    if codes is None:
+        codes = torch.empty((M, rot.K), dtype=torch.int8, device=X_bf16.device)
+    if scales is None:
+        scales = torch.empty((M,), dtype=torch.float32, device=X_bf16.device)
+    if workspace is None:
+        workspace = torch.empty((max(1, trdq_rotate_dense_workspace(rot, M)),), dtype=torch.uint8, device=X_bf16.device)
+    ldx = int(X_bf16.stride(0)) if M > 1 else rot.K
+    _check(lib().trdq_rotate_dense_quantize(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(codes), _ptr(scales), _ptr(workspace),
+                                            int(workspace.numel() * workspace.element_size()), _stream()),
+           "trdq_rotate_dense_quantize")
+    return codes, scales
+
+
+def trdq_greedy_rotation_block(x_calib, gauss) -> Tuple[np.ndarray, int]:
+    """(R fp32 [128,128], n) of Eq. 6-7 for one block; host only."""
+    x = np.ascontiguousarray(x_calib, dtype=np.float32)
+    g = np.ascontiguousarray(gauss, dtype=np.float64)
+    assert x.ndim == 2 and x.shape[1] == 128 and g.ndim == 3 and g.shape[1:] == (128, 128)
+    R = np.empty((128, 128), np.float32)
+    n = C.c_int32(0)
+    _check(lib().trdq_greedy_rotation_block(x.ctypes.data_as(C.POINTER(C.c_float)), int(x.shape[0]), int(g.shape[0]),
+                                            g.ctypes.data_as(C.POINTER(C.c_double)), R.ctypes.data_as(C.POINTER(C.c_float)),
+                                            C.byref(n)), "trdq_greedy_rotation_block")
+    return R, int(n.value)
 
 
 def trdq_linear(w: Weights, t: int, codes, scales, bias_bf16=None, out=None):

@@ -1,0 +1,212 @@
+"""GPU parity of the dense block rotations (Eq. 6-8) against the CPU oracle: online rotation on the tensor cores
+plus the per-token quantizer, the weight side through the exact block inverses, and the linear layer on both.
+
+Tolerance of the online side.  The oracle rounds the exact sum once; the tensor cores add 128 exact products in an
+unspecified order in fp32, so v may differ by a few units of 2^-24 * sum_i |x_i S_ij| (allowed here: 2^-20 times that
+sum).  Scales inherit that difference at the row maximum; a code may differ by one step only where the oracle's value
+before rounding lies within the propagated distance of a .5 boundary.  Whenever every partial sum is exactly
+representable (small integers times powers of two) the comparison is bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import trdq_oracle as O
+from paper_2503_06564_b200 import workloads as WL
+from tests.util import bf16_to_f32_np, check_output, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+ACC_TOL = 2.0 ** -20
+
+
+def orthogonal_blocks(G, nb, seed):
+    rng = np.random.default_rng(seed)
+    out = np.empty((G, nb, 128, 128), np.float32)
+    for g in range(G):
+        for b in range(nb):
+            q, r = np.linalg.qr(rng.standard_normal((128, 128)))
+            out[g, b] = (q * np.sign(np.diag(r))).astype(np.float32)
+    return out
+
+
+def sylvester(n=128):
+    H = np.ones((1, 1))
+    while H.shape[0] < n:
+        H = np.block([[H, H], [H, -H]])
+    return H
+
+
+def acts(M, K, seed):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((M, K))
+    x[:, rng.choice(K, max(1, K // 100), replace=False)] *= 30.0
+    return WL.to_bf16_bits(x)
+
+
+def check_dense_codes(codes, scales, x_bits, stored_bits):
+    """Compares GPU codes / scales with the oracle under the accumulation tolerance; returns the number of differing codes."""
+    K = x_bits.shape[1]
+    v = O.rotate_dense(x_bits, stored_bits)
+    c_ref, s_ref = O.quantize_rows(v)
+    x = np.abs(WL.bf16_bits_to_f32(x_bits).astype(np.float64))
+    S = np.abs(WL.bf16_bits_to_f32(stored_bits).astype(np.float64))
+    mass = np.concatenate([x[:, 128 * b:128 * (b + 1)] @ S[b] for b in range(K // 128)], axis=1)   # sum_i |x_i S_ij|
+    tol_v = ACC_TOL * mass
+    amax = np.abs(v).max(axis=1).astype(np.float64)
+    tol_amax = tol_v.max(axis=1)
+    assert np.all(np.abs(scales.astype(np.float64) - s_ref) <= tol_amax / 127.0 * 1.001 + 2.0 ** -23 * s_ref)
+    assert not np.any(codes == -128)
+    diff = codes.astype(np.int32) - c_ref
+    bad = diff != 0
+    if bad.any():
+        assert np.abs(diff).max() <= 1
+        safe = np.where(amax > 0, amax, 1.0)
+        inv = 127.0 / safe
+        u = v.astype(np.float64) * inv[:, None]
+        du = inv[:, None] * tol_v + 127.0 * (tol_amax / safe)[:, None] + 2.0 ** -15
+        dist = np.abs(u - np.floor(u) - 0.5)
+        assert np.all(dist[bad] <= du[bad]), "a differing code is not at a rounding boundary"
+        assert bad.sum() <= 2e-3 * codes.size, f"{bad.sum()} of {codes.size} codes differ"
+    return int(bad.sum())
+
+
+@pytest.mark.parametrize("M,K,G", [(300, 1152, 2), (129, 384, 1), (1, 128, 1), (1000, 4608, 1), (128, 256, 3), (77, 2048, 1)])
+def test_dense_codes_match_oracle(M, K, G):
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(7 + K)
+    blocks = orthogonal_blocks(G, K // 128, 100 + K)
+    smooth = rng.uniform(0.25, 4.0, (G, K)).astype(np.float32)
+    bounds = WL.group_bounds(G)
+    rot = trdq.DenseRotation(K, bounds, blocks, smooth)
+    x = acts(M, K, 5 + M)
+    xd = to_dev_bf16(x)
+    total_bad = 0
+    for g in range(G):
+        codes, scales = trdq.trdq_rotate_dense_quantize(rot, int(bounds[g]), xd)
+        stored = O.dense_stored_blocks(blocks[g], smooth[g])
+        total_bad += check_dense_codes(codes.cpu().numpy(), scales.cpu().numpy(), x, stored)
+    assert trdq.trdq_device_status() == 0
+    print(f"M={M} K={K}: {total_bad} of {G * M * K} codes off by one")
+
+
+def test_dense_rotation_exact_cases_are_bit_exact():
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(11)
+    K, M = 512, 261
+    H = sylvester()
+    perm = rng.permutation(128)
+    P = np.zeros((128, 128))
+    P[perm, np.arange(128)] = 1.0                            # (x P)[j] = x[perm[j]]
+    blocks = np.stack([H / 8.0, -H / 16.0, np.eye(128), P]).astype(np.float32)[None]
+    rot = trdq.DenseRotation(K, [0, 1000], blocks, None)
+    x = WL.to_bf16_bits(rng.integers(-12, 13, (M, K)).astype(np.float64))
+    x[5] = 0                                                 # an all-zero token: scale 0, codes 0
+    codes, scales = trdq.trdq_rotate_dense_quantize(rot, 10, to_dev_bf16(x))
+    stored = O.dense_stored_blocks(blocks[0], None)
+    v = O.rotate_dense(x, stored)
+    c_ref, s_ref = O.quantize_rows(v)
+    assert np.array_equal(scales.cpu().numpy(), s_ref) and np.array_equal(codes.cpu().numpy(), c_ref)
+    assert s_ref[5] == 0 and not c_ref[5].any()
+    # the Hadamard blocks reproduce the butterfly route, the identity and permutation blocks move values unchanged
+    xf = WL.bf16_bits_to_f32(x)
+    assert np.array_equal(v[:, :128], O.rotate(x[:, :128], np.full(128, 0.125, np.float32)))
+    assert np.array_equal(v[:, 256:384], xf[:, 256:384]) and np.array_equal(v[:, 384:], xf[:, 384:][:, perm])
+    # a strided input (row stride > K) and caller-provided buffers
+    wide = torch.zeros((M, K + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :K] = to_dev_bf16(x)
+    ws = torch.empty(trdq.trdq_rotate_dense_workspace(rot, M), dtype=torch.uint8, device="cuda")
+    c2, s2 = trdq.trdq_rotate_dense_quantize(rot, 10, wide[:, :K], workspace=ws)
+    assert torch.equal(c2, codes) and torch.equal(s2, scales)
+    assert trdq.trdq_device_status() == 0
+
+
+@pytest.mark.parametrize("wbits", [8, 4])
+def test_dense_prepared_weights_match_oracle(wbits):
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(21)
+    K, N, G = 384, 208, 2
+    blocks = orthogonal_blocks(G, K // 128, 31)
+    smooth = rng.uniform(0.25, 4.0, (G, K)).astype(np.float32)
+    w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.02)
+    rot = trdq.DenseRotation(K, WL.group_bounds(G), blocks, smooth)
+    w = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), wbits)
+    for g in range(G):
+        inv = O.invert_blocks(O.dense_stored_blocks(blocks[g], smooth[g]))
+        wr = O.prepare_dense_rotate(w_bits, inv)
+        codes, scales = w.view_tensors(g)
+        if wbits == 8:
+            c_ref, s_ref = O.quantize_rows(wr)
+        else:
+            c_ref, s_ref = O.quantize_w4_rows(wr)
+        # the two inverses come from separate fp64 eliminations: a last-bit difference may flip an fp32 rounding of wr
+        # once in many millions of values, so equality is expected and a handful of one-step differences tolerated
+        cg = codes.cpu().numpy()
+        if wbits == 8:
+            d = np.abs(cg.astype(np.int32) - c_ref)
+            assert d.max() <= 1 and (d != 0).sum() <= 2
+        else:
+            assert (cg != c_ref).sum() <= 2
+        assert np.allclose(scales.cpu().numpy(), s_ref, rtol=2.0 ** -22, atol=0)
+
+
+@pytest.mark.parametrize("M,K,N,wbits", [(384, 1152, 1152, 8), (200, 512, 272, 8), (256, 1152, 384, 4)])
+def test_dense_linear_end_to_end(M, K, N, wbits):
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(33 + N)
+    blocks = orthogonal_blocks(1, K // 128, 41 + K)
+    smooth = rng.uniform(0.5, 2.0, (1, K)).astype(np.float32)
+    x = acts(M, K, 17)
+    w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.02)
+    bias_bits = WL.to_bf16_bits(rng.standard_normal(N) * 0.01)
+    rot = trdq.DenseRotation(K, [0, 1000], blocks, smooth)
+    w = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), wbits)
+    codes, scales = trdq.trdq_rotate_dense_quantize(rot, 500, to_dev_bf16(x))
+    y = trdq.trdq_linear(w, 500, codes, scales, to_dev_bf16(bias_bits))
+    # the integer GEMM and the epilogue are exact functions of the codes: oracle on the codes the GPU produced
+    wq, sw = w.view_tensors(0)
+    rows = np.arange(0, M, max(1, M // 64), dtype=np.int64)
+    if wbits == 8:
+        y_ref = O.linear_w8_rows(codes.cpu().numpy(), scales.cpu().numpy(), wq.cpu().numpy(), sw.cpu().numpy(), bias_bits, rows)
+    else:
+        y_ref = O.linear_w4_rows(codes.cpu().numpy(), scales.cpu().numpy(), wq.cpu().numpy(), sw.cpu().numpy(), bias_bits, rows)
+    check_output(bf16_to_f32_np(y)[rows], y_ref)
+    # Eq. 9: the rotated, quantized layer still computes X W^T + bias (here to quantization accuracy)
+    xf = WL.bf16_bits_to_f32(x).astype(np.float64)
+    wf = WL.bf16_bits_to_f32(w_bits).astype(np.float64)
+    exact = xf @ wf.T + WL.bf16_bits_to_f32(bias_bits).astype(np.float64)
+    rel = np.linalg.norm(bf16_to_f32_np(y).astype(np.float64) - exact) / np.linalg.norm(exact)
+    assert rel < (0.03 if wbits == 8 else 0.2), rel
+    assert trdq.trdq_device_status() == 0
+
+
+def test_dense_rotation_argument_errors():
+    import torch
+    from paper_2503_06564_b200 import trdq
+    K = 256
+    blocks = orthogonal_blocks(1, 2, 3)
+    rot = trdq.DenseRotation(K, [0, 1000], blocks, None)
+    x = torch.zeros((64, K), dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_rotate_dense_quantize(rot, 0, x, workspace=small)
+    assert e.value.status == 8                                   # workspace too small
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_rotate_quantize(rot, 0, x)
+    assert e.value.status == 10                                  # the Hadamard call does not take dense blocks
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_rotate_dense_quantize(rot, 1000, x)
+    assert e.value.status == 4
+    had = trdq.Rotation(K, [0, 1000], np.ones((1, K), np.int8))
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_rotate_dense_quantize(had, 0, x, workspace=torch.empty(4096, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 10
+    singular = blocks.copy()
+    singular[0, 1, :, 9] = singular[0, 1, :, 4]
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.DenseRotation(K, [0, 1000], singular, None)
+    assert e.value.status == 5
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.DenseRotation(K, [0, 1000], blocks, np.zeros((1, K), np.float32))
+    assert e.value.status == 5
+    codes, scales = trdq.trdq_rotate_dense_quantize(rot, 0, x[:0])   # M = 0: nothing to do
+    assert codes.shape[0] == 0

@@ -116,3 +116,27 @@ def test_zigzag_permutation_matches_the_oracle_and_rejects_bad_input(lib):
     with pytest.raises(trdq.TrdqError) as e:
         trdq.Rotation(256, [0, 1000], np.ones((1, 256), np.int8), perm=np.zeros((1, 256), np.int32))
     assert e.value.status == 5
+
+
+def test_greedy_rotation_block_matches_oracle(lib):
+    """Eq. 6-7 on the host: the library's construction against the oracle's on the same calibration rows and draws."""
+    from oracle import trdq_oracle as O
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((48, 128)).astype(np.float32)
+    x[:, 17] *= 70.0
+    x[:, 101] *= 30.0
+    gauss = rng.standard_normal((5, 128, 128))
+    R, n = trdq.trdq_greedy_rotation_block(x, gauss)
+    R_ref, n_ref, trace = O.greedy_block(x.astype(np.float64), gauss)
+    assert n == n_ref
+    assert np.max(np.abs(R.astype(np.float64) - R_ref)) <= 2.0 ** -24 + 1e-9   # one rounding to fp32 of entries below 1
+    assert np.max(np.abs(R.astype(np.float64) @ R.astype(np.float64).T - np.eye(128))) < 1e-5
+    assert np.max(np.abs(x.astype(np.float64) @ R_ref)) < 0.2 * np.max(np.abs(x))
+    # argument errors are found on the host
+    assert lib.trdq_greedy_rotation_block(None, 4, 1, None, None, None) == 1
+    bad = x.copy()
+    bad[0, 0] = np.inf
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_greedy_rotation_block(bad, gauss)
+    assert e.value.status == 5
