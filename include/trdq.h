@@ -229,8 +229,8 @@ trdq_status trdq_rotation_create_dense(int32_t K, int32_t num_groups, const int3
 /* Online side with dense blocks: v[m, 128 b + j] = sum_i X[m, 128 b + i] * S_b[i][j] on the tensor cores (bf16 operands, every
  * product exact, fp32 accumulation), then the per-token quantizer of trdq_rotate_quantize on v (same scale and code
  * definitions).  The row maximum must be known before the first code, so X is read twice; `workspace` (device,
- * 4-byte aligned, at least the size trdq_rotate_dense_workspace reports = 4 * (K/128) * M bytes) holds the per-block row
- * maxima between the two passes.  It is scratch: no initialisation needed, contents undefined afterwards; two calls that
+ * 4-byte aligned, at least the size trdq_rotate_dense_workspace reports = 32 * M bytes) holds partial row maxima between
+ * the two passes.  It is scratch: no initialisation needed, contents undefined afterwards; two calls that
  * may overlap on the GPU need separate workspaces.  Asynchronous on `stream`; allocates nothing.
  * TRDQ_ERR_MISMATCH if rot was not made by trdq_rotation_create_dense; TRDQ_ERR_NOMEM if the workspace is too small;
  * otherwise the errors of trdq_rotate_quantize.  Because the accumulation order inside the tensor cores is not

@@ -9,16 +9,16 @@
 // per 16 input channels computes v exactly up to the accumulation order.
 //
 // The per-token scale needs the maximum of |v| over the WHOLE row before any code can be formed, and a
-// row of 128 tokens x K channels of fp32 does not fit in tensor memory (512 columns).  So the work is cut
-// the other way: a CTA owns ONE block column b (its S_b stays in shared memory for the whole kernel, so
-// matrix traffic is paid once) and walks down the token tiles; two passes over X:
-//   pass 0  v = X_tile S_b on the tensor cores, per-row maximum of |v| -> partial[b][m]
-//   pass 1  the same product again (bit-identical: same instructions, same operands), row maximum =
-//           max over the K/128 partials, codes = rne(v * fl(127 / amax)), written through TMA stores.
-// The second pass walks the tiles in the opposite order, so what the first pass read last is still in L2.
-// Both passes run the same warp-specialised pipeline: warp 0 streams X tiles with TMA into a four-stage
-// ring, warp 1 issues the MMAs into one of four 128-column accumulators, eight warps drain them.
-// Every wait is bounded.
+// tile of 128 tokens x K channels of fp32 does not fit in tensor memory (512 columns).  So X is read twice:
+//   pass 0 (amax)      a CTA owns token tiles and walks across the K/128 blocks; X tile and S_b arrive together
+//                      through a three-stage ring (S comes from L2, X from HBM); the drain warps keep a running
+//                      per-row maximum of |v| in registers and write amax[m] once per row.
+//   pass 1 (quantize)  a CTA owns ONE block column b (S_b stays in shared memory, so matrix traffic is paid once)
+//                      and walks down the token tiles in the opposite order of pass 0, so that what was read
+//                      last is still in L2; the product is formed again (bit-identical: same instructions on
+//                      the same operands), codes = rne(v * fl(127 / amax)), written through TMA stores.
+// Both passes are warp specialised: warp 0 issues TMA loads, warp 1 the MMAs into one of four 128-column
+// accumulators, warp 2 owns tensor memory, warps 4.. drain.  Every wait is bounded.
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -29,30 +29,37 @@
 namespace trdq {
 namespace {
 
-constexpr int kRows = 128;                      // token rows per tile = M of the MMA
-constexpr int kStages = 4;                      // X tiles in flight
+constexpr int kRows = 128;                          // token rows per tile = M of the MMA
 constexpr int kTileBytes = kRows * TRDQ_BLOCK * 2;  // 128 x 128 bf16: two swizzle atoms of 128 rows x 64 columns
 constexpr int kAtomBytes = kTileBytes / 2;
 constexpr int kAccSlots = 4;
 constexpr int kAccCols = TRDQ_BLOCK;
 constexpr int kTmemCols = 512;
-constexpr int kThreads = 384;                   // warp 0 TMA, warp 1 MMA, warp 2 tensor-memory owner, warps 4-11 drain
-constexpr int kDrainWarps = 8;
-constexpr int kOutStageBytes = kDrainWarps * 2 * 2048;  // per warp two tiles of 32 rows x 64 codes
+constexpr int kThreads = 384;                       // warp 0 TMA, warp 1 MMA, warp 2 tensor-memory owner, warps 4-11 drain
 constexpr int kBarrierBytes = 256;
-constexpr int kSmemBytes = 1024 + kTileBytes + kStages * kTileBytes + kOutStageBytes + kBarrierBytes;
-constexpr float kRoundMagic = 12582912.0f;      // 1.5 * 2^23: adding it leaves rne(u) in the low mantissa bits
+// pass 0: ring of (X tile, S_b) pairs
+constexpr int kStages0 = 3;
+constexpr int kSmemBytes0 = 1024 + kStages0 * 2 * kTileBytes + kBarrierBytes;
+// pass 1: resident S_b, ring of X tiles, per drain warp two staging tiles of 32 rows x 64 codes
+constexpr int kStages1 = 4;
+constexpr int kDrainWarps1 = 8;
+constexpr int kOutStageBytes = kDrainWarps1 * 2 * 2048;
+constexpr int kSmemBytes1 = 1024 + kTileBytes + kStages1 * kTileBytes + kOutStageBytes + kBarrierBytes;
+constexpr float kRoundMagic = 12582912.0f;          // 1.5 * 2^23: adding it leaves rne(u) in the low mantissa bits
 
 struct alignas(64) DenseParams {
   CUtensorMap tmap_x;      // bf16 [M, K] (row stride ldx), box 64 columns x 128 rows, 128-byte swizzle
   CUtensorMap tmap_s;      // bf16 [G * K/128 * 128, 128]: S_b transposed (row j = output channel), same box
   CUtensorMap tmap_codes;  // int8 [M, K], box 64 x 32, 64-byte swizzle
-  float* partial;          // [K/128][M]: per block and row, max |v|
+  float* amax;             // [splits][M]: max of |v| over the row's blocks of each split
   float* scales;           // [M]
-  int32_t M, K, tiles_m;
+  int32_t M, K;
+  int32_t tile_begin, tile_end;      // token tiles of this launch
+  int32_t splits, blocks_per_split;  // pass 0 cuts the K/128 blocks into `splits` ranges when there are few token tiles
   int32_t s_row0;          // first row of this group's matrices in tmap_s
   uint32_t* status;
 };
+constexpr int kMaxSplits = 8;
 
 // kind::f16 instruction descriptor: bf16 A and B, both K-major, fp32 D, M = 128, N = 128.
 constexpr uint32_t kIdescBf16 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TRDQ_BLOCK >> 3) << 17) |
@@ -68,35 +75,175 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       : "memory");
 }
 
-template <int PASS>
-__global__ void __launch_bounds__(kThreads, 1) rotate_dense_kernel(const __grid_constant__ DenseParams p) {
+// One 128 x 128 x 128 product: X tile (two atoms) times S_b (two atoms) into the accumulator at d_tmem.
+__device__ __forceinline__ void mma_tile(uint32_t d_tmem, uint32_t x_addr, uint32_t s_addr) {
+#pragma unroll
+  for (int a = 0; a < 2; ++a) {
+    const uint64_t a_desc = umma_desc_k_sw128(x_addr + a * kAtomBytes);
+    const uint64_t b_desc = umma_desc_k_sw128(s_addr + a * kAtomBytes);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)  // 16 input channels = 32 bytes along K = +2 in the 16-byte address field
+      umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, (a | k) != 0 ? 1u : 0u);
+  }
+}
+
+struct Pipe {
+  int idx = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance(int n) {
+    if (++idx == n) {
+      idx = 0;
+      phase ^= 1;
+    }
+  }
+};
+
+// ------------------------------------------------------------------------------ pass 0 ----
+__global__ void __launch_bounds__(kThreads, 1) rotate_dense_amax_kernel(const __grid_constant__ DenseParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t s_tile = smem_base;                            // S_b, resident
-  const uint32_t x_ring = smem_base + kTileBytes;               // kStages tiles
-  const uint32_t out_stage_base = x_ring + kStages * kTileBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes + kStages * kTileBytes + kOutStageBytes);
-  const uint32_t bar_full = smem_u32(bars);            // [kStages]
-  const uint32_t bar_empty = bar_full + 8 * kStages;   // [kStages]
-  const uint32_t bar_tfull = bar_empty + 8 * kStages;  // [kAccSlots]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages0 * 2 * kTileBytes);
+  const uint32_t bar_full = smem_u32(bars);             // [kStages0]
+  const uint32_t bar_empty = bar_full + 8 * kStages0;   // [kStages0]
+  const uint32_t bar_tfull = bar_empty + 8 * kStages0;  // [kAccSlots]
   const uint32_t bar_tempty = bar_tfull + 8 * kAccSlots;
-  const uint32_t bar_s = bar_tempty + 8 * kAccSlots;   // S_b has landed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccSlots + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages0 + 2 * kAccSlots);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int b = blockIdx.y;                            // block column of this CTA
-  constexpr int kDrainArrivals = PASS == 0 ? 4 : 8;    // pass 0 drains with one warp per lane quarter
+  const int b_begin = blockIdx.y * p.blocks_per_split;
+  const int b_end = min(p.K / TRDQ_BLOCK, b_begin + p.blocks_per_split);
+  const int tile_first = p.tile_begin + blockIdx.x;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kStages0; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
     for (int a = 0; a < kAccSlots; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, kDrainArrivals);
+      mbar_init(bar_tempty + 8 * a, 4);  // one drain warp per lane quarter
+    }
+    fence_mbar_init();
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&p.tmap_x);
+    prefetch_tensormap(&p.tmap_s);
+  }
+  griddep_launch_dependents();
+  griddep_wait();  // X comes from the kernel before; amax may still be read by it
+
+  if (warp == 0) {
+    if (elect_one()) {
+      BoundedWaiter w(p.status, kStatusTimeoutProducer);
+      Pipe st;
+      for (int tile = tile_first; tile < p.tile_end; tile += gridDim.x)
+        for (int b = b_begin; b < b_end; ++b) {
+          w.wait(bar_empty + 8 * st.idx, st.phase ^ 1);
+          const uint32_t dst = smem_base + st.idx * 2 * kTileBytes;
+          const uint32_t bar = bar_full + 8 * st.idx;
+          mbar_arrive_expect_tx(bar, 2 * kTileBytes);
+          tma_load_2d(dst, &p.tmap_x, b * TRDQ_BLOCK, tile * kRows, bar);  // rows >= M read as zero
+          tma_load_2d(dst + kAtomBytes, &p.tmap_x, b * TRDQ_BLOCK + 64, tile * kRows, bar);
+          tma_load_2d(dst + kTileBytes, &p.tmap_s, 0, p.s_row0 + b * TRDQ_BLOCK, bar);
+          tma_load_2d(dst + kTileBytes + kAtomBytes, &p.tmap_s, 64, p.s_row0 + b * TRDQ_BLOCK, bar);
+          st.advance(kStages0);
+        }
+      w.settle();
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      BoundedWaiter w(p.status, kStatusTimeoutMma);
+      Pipe st, acc;
+      for (int tile = tile_first; tile < p.tile_end; tile += gridDim.x)
+        for (int b = b_begin; b < b_end; ++b) {
+          w.wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1);
+          w.wait(bar_full + 8 * st.idx, st.phase);
+          tc_fence_after();
+          const uint32_t x_addr = smem_base + st.idx * 2 * kTileBytes;
+          mma_tile(tmem_base + acc.idx * kAccCols, x_addr, x_addr + kTileBytes);
+          umma_commit(bar_empty + 8 * st.idx);
+          umma_commit(bar_tfull + 8 * acc.idx);
+          st.advance(kStages0);
+          acc.advance(kAccSlots);
+        }
+      w.settle();
+    }
+  } else if (warp >= 4 && warp < 8) {
+    const int q = warp & 3;  // the lane quarter of tensor memory this warp may read
+    BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
+    Pipe acc;
+    for (int tile = tile_first; tile < p.tile_end; tile += gridDim.x) {
+      const int row = tile * kRows + q * 32 + lane;
+      float mx = 0.0f;
+      for (int b = b_begin; b < b_end; ++b) {
+        w.wait(bar_tfull + 8 * acc.idx, acc.phase);
+        __syncwarp();
+        tc_fence_after();
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc.idx * kAccCols;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(t_row + c * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(__uint_as_float(r[j])));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * acc.idx);
+        acc.advance(kAccSlots);
+      }
+      if (row < p.M) p.amax[static_cast<size_t>(blockIdx.y) * p.M + row] = mx;
+    }
+    w.settle();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------ pass 1 ----
+__global__ void __launch_bounds__(kThreads, 1) rotate_dense_quantize_kernel(const __grid_constant__ DenseParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t s_tile = smem_base;                            // S_b, resident
+  const uint32_t x_ring = smem_base + kTileBytes;
+  const uint32_t out_stage_base = x_ring + kStages1 * kTileBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes + kStages1 * kTileBytes + kOutStageBytes);
+  const uint32_t bar_full = smem_u32(bars);             // [kStages1]
+  const uint32_t bar_empty = bar_full + 8 * kStages1;   // [kStages1]
+  const uint32_t bar_tfull = bar_empty + 8 * kStages1;  // [kAccSlots]
+  const uint32_t bar_tempty = bar_tfull + 8 * kAccSlots;
+  const uint32_t bar_s = bar_tempty + 8 * kAccSlots;    // S_b has landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages1 + 2 * kAccSlots + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.y;  // block column of this CTA
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages1; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < kAccSlots; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, kDrainWarps1);
     }
     mbar_init(bar_s, 1);
     fence_mbar_init();
@@ -112,153 +259,112 @@ __global__ void __launch_bounds__(kThreads, 1) rotate_dense_kernel(const __grid_
   if (threadIdx.x == 0) {
     prefetch_tensormap(&p.tmap_x);
     prefetch_tensormap(&p.tmap_s);
-    if (PASS == 1) prefetch_tensormap(&p.tmap_codes);
+    prefetch_tensormap(&p.tmap_codes);
     // the matrices are constants of the rotation object: they may be fetched while the kernel before still runs
     mbar_arrive_expect_tx(bar_s, kTileBytes);
     tma_load_2d(s_tile, &p.tmap_s, 0, p.s_row0 + b * TRDQ_BLOCK, bar_s);
     tma_load_2d(s_tile + kAtomBytes, &p.tmap_s, 64, p.s_row0 + b * TRDQ_BLOCK, bar_s);
   }
   griddep_launch_dependents();
-  griddep_wait();  // X (and in pass 1 the partial maxima) come from the kernel before; the code buffer may still be read by it
+  griddep_wait();  // X and the row maxima come from the kernels before; the code buffer may still be read by them
 
-  // Tile order: pass 0 ascending, pass 1 descending (what pass 0 touched last is the likeliest to be in L2).
-  const int my_tiles = blockIdx.x < p.tiles_m ? (p.tiles_m - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
-  auto tile_row0 = [&](int it) {
-    const int t = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
-    return (PASS == 0 ? t : p.tiles_m - 1 - t) * kRows;
-  };
+  // This CTA's tiles, from the last token tile of the launch backwards.
+  const int tiles = p.tile_end - p.tile_begin;
+  const int my_tiles = static_cast<int>(blockIdx.x) < tiles ? (tiles - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+  auto tile_row0 = [&](int it) { return (p.tile_end - 1 - (static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x))) * kRows; };
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
       BoundedWaiter w(p.status, kStatusTimeoutProducer);
-      int stage = 0;
-      uint32_t phase = 0;
+      Pipe st;
       for (int it = 0; it < my_tiles; ++it) {
         const int row0 = tile_row0(it);
-        w.wait(bar_empty + 8 * stage, phase ^ 1);
-        const uint32_t dst = x_ring + stage * kTileBytes;
-        mbar_arrive_expect_tx(bar_full + 8 * stage, kTileBytes);
-        tma_load_2d(dst, &p.tmap_x, b * TRDQ_BLOCK, row0, bar_full + 8 * stage);  // rows >= M read as zero
-        tma_load_2d(dst + kAtomBytes, &p.tmap_x, b * TRDQ_BLOCK + 64, row0, bar_full + 8 * stage);
-        if (++stage == kStages) {
-          stage = 0;
-          phase ^= 1;
-        }
+        w.wait(bar_empty + 8 * st.idx, st.phase ^ 1);
+        const uint32_t dst = x_ring + st.idx * kTileBytes;
+        mbar_arrive_expect_tx(bar_full + 8 * st.idx, kTileBytes);
+        tma_load_2d(dst, &p.tmap_x, b * TRDQ_BLOCK, row0, bar_full + 8 * st.idx);
+        tma_load_2d(dst + kAtomBytes, &p.tmap_x, b * TRDQ_BLOCK + 64, row0, bar_full + 8 * st.idx);
+        st.advance(kStages1);
       }
       w.settle();
     }
   } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
     if (elect_one()) {
       BoundedWaiter w(p.status, kStatusTimeoutMma);
       w.wait(bar_s, 0);
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
+      Pipe st, acc;
       for (int it = 0; it < my_tiles; ++it) {
-        w.wait(bar_tempty + 8 * acc, acc_phase ^ 1);
-        w.wait(bar_full + 8 * stage, phase);
+        w.wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1);
+        w.wait(bar_full + 8 * st.idx, st.phase);
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * kAccCols;
-        const uint32_t x_addr = x_ring + stage * kTileBytes;
-#pragma unroll
-        for (int a = 0; a < 2; ++a) {
-          const uint64_t a_desc = umma_desc_k_sw128(x_addr + a * kAtomBytes);
-          const uint64_t b_desc = umma_desc_k_sw128(s_tile + a * kAtomBytes);
-#pragma unroll
-          for (int k = 0; k < 4; ++k)  // 16 input channels = 32 bytes along K = +2 in the 16-byte address field
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, (a | k) != 0 ? 1u : 0u);
-        }
-        umma_commit(bar_empty + 8 * stage);
-        umma_commit(bar_tfull + 8 * acc);
-        if (++stage == kStages) {
-          stage = 0;
-          phase ^= 1;
-        }
-        if (++acc == kAccSlots) {
-          acc = 0;
-          acc_phase ^= 1;
-        }
+        mma_tile(tmem_base + acc.idx * kAccCols, x_ring + st.idx * kTileBytes, s_tile);
+        umma_commit(bar_empty + 8 * st.idx);
+        umma_commit(bar_tfull + 8 * acc.idx);
+        st.advance(kStages1);
+        acc.advance(kAccSlots);
       }
       w.settle();
     }
-  } else if (warp >= 4 && (PASS == 1 || warp < 8)) {
-    // ------------------------------------------------------------------- drain
+  } else if (warp >= 4) {
     const int ew = warp - 4;
     const int q = ew & 3;      // = warp % 4: the lane quarter of tensor memory this warp may read
-    const int half = ew >> 2;  // pass 1: which 64 of the 128 columns
-    const int nb = p.K / TRDQ_BLOCK;
+    const int half = ew >> 2;  // which 64 of the 128 columns
     const uint32_t my_stage = out_stage_base + ew * 4096;
     BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
-    int acc = 0;
-    uint32_t acc_phase = 0;
+    Pipe acc;
+    // the row maxima of the next tile are fetched while the current one is drained (raw values are kept in
+    // registers and only combined one iteration later, so that the loads never stall this warp)
+    float part[kMaxSplits];
+    auto fetch = [&](int it) {
+      const int row = tile_row0(it) + q * 32 + lane;
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) part[s] = (s < p.splits && row < p.M) ? __ldg(p.amax + static_cast<size_t>(s) * p.M + row) : 0.0f;
+    };
+    if (my_tiles > 0) fetch(0);
     for (int it = 0; it < my_tiles; ++it) {
       const int row0 = tile_row0(it);
       const int row = row0 + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      float inv = 0.0f;
-      if (PASS == 1) {
-        float amax = 0.0f;
-        if (row_ok)
-          for (int bb = 0; bb < nb; ++bb) amax = fmaxf(amax, __ldg(p.partial + static_cast<size_t>(bb) * p.M + row));
-        if (row_ok && b == 0 && half == 0) p.scales[row] = __fdiv_rn(amax, 127.0f);
-        inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-      }
-      w.wait(bar_tfull + 8 * acc, acc_phase);
+      float amax = part[0];
+#pragma unroll
+      for (int s = 1; s < kMaxSplits; ++s) amax = fmaxf(amax, part[s]);
+      if (it + 1 < my_tiles) fetch(it + 1);
+      if (row < p.M && b == 0 && half == 0) p.scales[row] = __fdiv_rn(amax, 127.0f);
+      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+      w.wait(bar_tfull + 8 * acc.idx, acc.phase);
       __syncwarp();
       tc_fence_after();
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols;
-      if (PASS == 0) {
-        float mx = 0.0f;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld_32x32(t_row + c * 32, r);
-          tmem_wait_ld();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc.idx * kAccCols + half * 64;
+      const uint32_t tile_smem = my_stage + (it & 1) * 2048;
+      if (lane == 0) bulk_wait_group_read<1>();  // the store issued two tiles ago has finished reading this buffer
+      __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(__uint_as_float(r[j])));
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(t_row + c * 32, r);
+        tmem_wait_ld();
+        uint32_t wds[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint32_t by[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) by[e] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r[4 * j + e]), inv), kRoundMagic));
+          wds[j] = __byte_perm(__byte_perm(by[0], by[1], 0x0040), __byte_perm(by[2], by[3], 0x0040), 0x5410);
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
-        if (row_ok) p.partial[static_cast<size_t>(b) * p.M + row] = mx;
-      } else {
-        const uint32_t tile_smem = my_stage + (it & 1) * 2048;
-        if (lane == 0) bulk_wait_group_read<1>();  // the store issued two tiles ago has finished reading this buffer
-        __syncwarp();
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld_32x32(t_row + half * 64 + c * 32, r);
-          tmem_wait_ld();
-          uint32_t wds[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            uint32_t by[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              by[e] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r[4 * j + e]), inv), kRoundMagic));
-            wds[j] = __byte_perm(__byte_perm(by[0], by[1], 0x0040), __byte_perm(by[2], by[3], 0x0040), 0x5410);
-          }
-          // staging tile: row = lane, 64 bytes per row, 16-byte chunk v stored at v ^ ((lane >> 1) & 3)
-          st_shared_v4(tile_smem + lane * 64 + (((2 * c) ^ ((lane >> 1) & 3)) << 4), wds[0], wds[1], wds[2], wds[3]);
-          st_shared_v4(tile_smem + lane * 64 + (((2 * c + 1) ^ ((lane >> 1) & 3)) << 4), wds[4], wds[5], wds[6], wds[7]);
-        }
-        tc_fence_before();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar_tempty + 8 * acc);
-          tma_store_2d(&p.tmap_codes, b * TRDQ_BLOCK + half * 64, row0 + q * 32, tile_smem);  // rows >= M are clipped
-          bulk_commit_group();
-        }
+        // staging tile: row = lane, 64 bytes per row, 16-byte chunk v stored at v ^ ((lane >> 1) & 3)
+        st_shared_v4(tile_smem + lane * 64 + (((2 * c) ^ ((lane >> 1) & 3)) << 4), wds[0], wds[1], wds[2], wds[3]);
+        st_shared_v4(tile_smem + lane * 64 + (((2 * c + 1) ^ ((lane >> 1) & 3)) << 4), wds[4], wds[5], wds[6], wds[7]);
       }
-      if (++acc == kAccSlots) {
-        acc = 0;
-        acc_phase ^= 1;
+      tc_fence_before();
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar_tempty + 8 * acc.idx);
+        tma_store_2d(&p.tmap_codes, b * TRDQ_BLOCK + half * 64, row0 + q * 32, tile_smem);  // rows >= M are clipped
+        bulk_commit_group();
       }
+      acc.advance(kAccSlots);
     }
-    if (PASS == 1 && lane == 0) bulk_wait_group_read<0>();
+    if (lane == 0) bulk_wait_group_read<0>();
     w.settle();
   }
 
@@ -353,23 +459,23 @@ __global__ void __launch_bounds__(256) quantize_rows_w4_kernel(const float* __re
   *reinterpret_cast<uint16_t*>(packed + grp * (TRDQ_BLOCK / 2) + 2 * lane) = two;
 }
 
-template <int PASS>
-cudaError_t launch_pass(const DenseParams& p, dim3 grid, cudaStream_t stream) {
-  static bool configured[16] = {};
+template <typename Kernel>
+cudaError_t launch_pass(Kernel kernel, int smem_bytes, bool* configured, const DenseParams& p, dim3 grid, cudaStream_t stream) {
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 16 && !configured[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(rotate_dense_kernel<PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  return launch_overlapped(rotate_dense_kernel<PASS>, grid, dim3(kThreads), kSmemBytes, stream, p);
+  return launch_overlapped(kernel, grid, dim3(kThreads), smem_bytes, stream, p);
 }
 
 }  // namespace
 
 uint64_t rotate_dense_workspace_bytes(int32_t M, int32_t K) {
-  return static_cast<uint64_t>(K / TRDQ_BLOCK) * static_cast<uint64_t>(M) * sizeof(float);
+  (void)K;
+  return static_cast<uint64_t>(kMaxSplits) * static_cast<uint64_t>(M) * sizeof(float);
 }
 
 trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const void* x_bf16, int64_t ldx, int32_t M, int8_t* codes,
@@ -381,22 +487,32 @@ trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const 
   p.tmap_s = rot->tmap_dense;
   st = encode_tmap_2d(&p.tmap_codes, codes, 1, K, M, K, 64, 32, 64);
   if (st != TRDQ_OK) return st;
-  p.partial = workspace;
+  p.amax = workspace;
   p.scales = scales;
   p.M = M;
   p.K = K;
-  p.tiles_m = (M + kRows - 1) / kRows;
   p.s_row0 = g * nb * TRDQ_BLOCK;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return TRDQ_ERR_CUDA;
-  // one CTA per SM: every block column gets the same number of CTAs, each walking its share of the token tiles
-  const int per_column = std::max(1, std::min(p.tiles_m, sms / nb));
-  const dim3 grid(per_column, nb);
-  if (launch_pass<0>(p, grid, stream) != cudaSuccess) return TRDQ_ERR_CUDA;
-  if (launch_pass<1>(p, grid, stream) != cudaSuccess) return TRDQ_ERR_CUDA;
+  static bool configured0[16] = {}, configured1[16] = {};
+  // Both passes cover all token tiles in one launch each.  (Cutting the rows into L2-sized chunks, each with its own
+  // pair of launches, was measured: the second read then hits L2, but the extra launches cost what the hits save.)
+  const int tiles = (M + kRows - 1) / kRows;
+  p.tile_begin = 0;
+  p.tile_end = tiles;
+  // pass 0: CTAs over the token tiles; with few tiles the blocks are cut into ranges so that the SMs are filled
+  p.splits = std::max(1, std::min({kMaxSplits, nb, sms / tiles}));
+  p.blocks_per_split = (nb + p.splits - 1) / p.splits;
+  p.splits = (nb + p.blocks_per_split - 1) / p.blocks_per_split;
+  if (launch_pass(rotate_dense_amax_kernel, kSmemBytes0, configured0, p, dim3(std::min(tiles, sms), p.splits), stream) != cudaSuccess)
+    return TRDQ_ERR_CUDA;
+  // pass 1: every block column gets the same number of CTAs, each walking its share of the token tiles
+  const int per_column = std::max(1, std::min(tiles, sms / nb));
+  if (launch_pass(rotate_dense_quantize_kernel, kSmemBytes1, configured1, p, dim3(per_column, nb), stream) != cudaSuccess)
+    return TRDQ_ERR_CUDA;
   return TRDQ_OK;
 }
 

@@ -210,3 +210,26 @@ def test_dense_rotation_argument_errors():
     assert e.value.status == 5
     codes, scales = trdq.trdq_rotate_dense_quantize(rot, 0, x[:0])   # M = 0: nothing to do
     assert codes.shape[0] == 0
+
+
+def test_dense_rotation_full_size_sampled_rows():
+    """The size the benchmark workloads use (M = 16384 tokens, hidden 1152), in the launch configuration a user gets:
+    the oracle evaluates a sample of rows, each row being independent of the others."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    M, K = 16384, 1152
+    blocks = orthogonal_blocks(1, K // 128, 77)
+    smooth = np.random.default_rng(78).uniform(0.5, 2.0, (1, K)).astype(np.float32)
+    rot = trdq.DenseRotation(K, [0, 1000], blocks, smooth)
+    torch.manual_seed(5)
+    xd = torch.randn((M, K), device="cuda")
+    xd[:, ::97] *= 25.0
+    xd = xd.to(torch.bfloat16)
+    codes, scales = trdq.trdq_rotate_dense_quantize(rot, 0, xd)
+    rows = np.unique(np.concatenate([np.arange(0, M, 61), [M - 1, M - 127, M - 128, M - 129]]))
+    x_rows = xd[torch.from_numpy(rows).cuda()].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    idx = torch.from_numpy(rows).cuda()
+    stored = O.dense_stored_blocks(blocks[0], smooth[0])
+    bad = check_dense_codes(codes[idx].cpu().numpy(), scales[idx].cpu().numpy(), x_rows, stored)
+    assert trdq.trdq_device_status() == 0
+    print(f"full size: {bad} of {rows.size * K} sampled codes off by one")
