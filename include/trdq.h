@@ -212,6 +212,19 @@ trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const
 trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
                              int32_t M, const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
 
+/* trdq_linear with the activation that follows the layer folded into its epilogue, so that the activation costs no
+ * pass over memory of its own (the first MLP linear of a transformer block is followed by GELU, and its output is what
+ * the next trdq_rotate_quantize reads):
+ *   y[m,n] = bf16( act( acc[m,n] * sx[m] * sw[n] + bias[n] ) )
+ * act: TRDQ_ACT_NONE (identical to trdq_linear) or TRDQ_ACT_GELU_TANH,
+ *   gelu(x) = 0.5 x (1 + tanh( sqrt(2/pi) (x + 0.044715 x^3) )),
+ * evaluated in fp32 with a relative error near 1e-6 (well inside the bf16 rounding of the result).  8- and 4-bit weights.
+ * The paper does not discuss activations; this is a fusion on the boundary of its layer.  Any other act: TRDQ_ERR_SHAPE. */
+#define TRDQ_ACT_NONE 0
+#define TRDQ_ACT_GELU_TANH 1
+trdq_status trdq_linear_act(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M, const void* bias_bf16,
+                            void* Y_bf16, int64_t ldy, int32_t act, void* stream);
+
 /* Dense block rotations (Sec. 3.2, Eq. 6-8): R = BlockDiag(R_b1 .. R_bK) with dense 128 x 128 orthogonal blocks, one
  * set per time-step group (Eq. 10).  blocks: host fp32 [G][K/128][128][128], R_b[i][j] with i the input channel
  * (v = x R).  smooth: host [G][K] (> 0) or NULL, the multiplier Delta_t of Eq. 10, folded into the rows of each block.
@@ -263,12 +276,16 @@ typedef struct trdq_layer_op {
   const void* bias_bf16;    /* dev [N] or NULL */
   void* Y_bf16;             /* dev [M, ldy] */
   int64_t ldy;
+  int32_t act;              /* TRDQ_ACT_NONE or TRDQ_ACT_GELU_TANH: activation folded into this layer's epilogue */
 } trdq_layer_op;
 
 /* Runs `count` layer ops in order for time-step t on `stream`: the group switch of the sampling
  * loop (Sec. 3.2: every layer selects its parameter set by the current time-step) without one
  * host round trip per kernel.  Validates every op before launching anything.  TRDQ_ERR_MISMATCH
- * if an op's rot and w disagree in K or in their time-step bounds. */
+ * if an op's rot and w disagree in K or in their time-step bounds.
+ * Every op has its own row count M, so a block whose unconditional branch reuses the conditional
+ * attention (attention sharing, Sec. 3.3) lists its attention linears with the conditional rows only
+ * and its MLP linears with all rows; nothing is computed for the skipped rows. */
 trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, void* stream);
 
 /* Raw accumulators of the integer GEMM (wbits = 8 only): acc[m, n] = sum_k q[m,k] * qw_g[n,k],

@@ -140,6 +140,17 @@ float quantize_span_asym(const float* v, int n, uint8_t* q, int32_t* zero_point)
   return scale;
 }
 
+// GELU in its tanh form (the activation between the two MLP linears of a DiT block), in double:
+//   gelu(x) = 0.5 x (1 + tanh(u)),  u = sqrt(2/pi) (x + 0.044715 x^3).
+// Written through the identity 0.5 (1 + tanh(u)) = 1 / (1 + exp(-2u)): the printed form loses all digits to the
+// cancellation in 1 + tanh(u) once u < -18 (x < -7) even in double, this one is accurate on both tails.
+// The paper does not discuss activations; this backs the fused-epilogue variant of the linear layer.
+inline double gelu_tanh(double x) {
+  const double c = 0.7978845608028654;  // sqrt(2/pi)
+  const double u = c * (x + 0.044715 * x * x * x);
+  return x / (1.0 + std::exp(-2.0 * u));
+}
+
 }  // namespace
 
 extern "C" {
@@ -249,8 +260,9 @@ void oracle_epilogue(const int32_t* acc, const float* sx, const float* sw, const
 }
 
 // W8A8 linear on a row subset: rows[i] selects the token; y is [num_rows, N].
-void oracle_linear_w8_rows(const int8_t* q, const float* sx, const int8_t* qw, const float* sw, const uint16_t* bias_bf16,
-                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+// act: 0 = none, 1 = GELU (tanh form) applied to the double value before the single rounding to fp32.
+void oracle_linear_w8_rows_act(const int8_t* q, const float* sx, const int8_t* qw, const float* sw, const uint16_t* bias_bf16,
+                               const int64_t* rows, int num_rows, int N, int K, int act, float* y) {
 #pragma omp parallel for schedule(static)
   for (int i = 0; i < num_rows; ++i) {
     const int64_t m = rows[i];
@@ -260,16 +272,21 @@ void oracle_linear_w8_rows(const int8_t* q, const float* sx, const int8_t* qw, c
         s += static_cast<int32_t>(q[m * K + k]) * static_cast<int32_t>(qw[static_cast<int64_t>(n) * K + k]);
       double r = static_cast<double>(s) * static_cast<double>(sx[m]) * static_cast<double>(sw[n]);
       if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      if (act == 1) r = gelu_tanh(r);
       y[static_cast<int64_t>(i) * N + n] = static_cast<float>(r);
     }
   }
+}
+void oracle_linear_w8_rows(const int8_t* q, const float* sx, const int8_t* qw, const float* sw, const uint16_t* bias_bf16,
+                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+  oracle_linear_w8_rows_act(q, sx, qw, sw, bias_bf16, rows, num_rows, N, K, 0, y);
 }
 
 // W4A8 linear on a row subset.  Every 128-wide k group has its own exact int32
 // partial sum, scaled by that group's weight scale:
 //   y = sx[m] * sum_kg (acc_kg * sw4[n, kg]) + bias[n]     (double, rounded once)
-void oracle_linear_w4_rows(const int8_t* q, const float* sx, const uint8_t* packed, const float* sw4, const uint16_t* bias_bf16,
-                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+void oracle_linear_w4_rows_act(const int8_t* q, const float* sx, const uint8_t* packed, const float* sw4, const uint16_t* bias_bf16,
+                               const int64_t* rows, int num_rows, int N, int K, int act, float* y) {
   const int groups = K / kBlock;
 #pragma omp parallel for schedule(static)
   for (int i = 0; i < num_rows; ++i) {
@@ -288,9 +305,14 @@ void oracle_linear_w4_rows(const int8_t* q, const float* sx, const uint8_t* pack
       }
       double r = static_cast<double>(sx[m]) * total;
       if (bias_bf16) r += static_cast<double>(bf16_to_float(bias_bf16[n]));
+      if (act == 1) r = gelu_tanh(r);
       y[static_cast<int64_t>(i) * N + n] = static_cast<float>(r);
     }
   }
+}
+void oracle_linear_w4_rows(const int8_t* q, const float* sx, const uint8_t* packed, const float* sw4, const uint16_t* bias_bf16,
+                           const int64_t* rows, int num_rows, int N, int K, float* y) {
+  oracle_linear_w4_rows_act(q, sx, packed, sw4, bias_bf16, rows, num_rows, N, K, 0, y);
 }
 
 // ---- fp64 cross-check path (structurally different from the butterfly) -------

@@ -128,7 +128,7 @@ def epilogue(acc, sx, sw, bias_bits=None) -> np.ndarray:
     return y
 
 
-def linear_w8_rows(q, sx, qw, sw, bias_bits, rows) -> np.ndarray:
+def linear_w8_rows(q, sx, qw, sw, bias_bits, rows, act: int = 0) -> np.ndarray:
     q = _c(q, np.int8)
     qw = _c(qw, np.int8)
     rows = _c(rows, np.int64)
@@ -136,12 +136,12 @@ def linear_w8_rows(q, sx, qw, sw, bias_bits, rows) -> np.ndarray:
     N = qw.shape[0]
     b = None if bias_bits is None else _c(bias_bits, np.uint16)
     y = np.empty((rows.size, N), np.float32)
-    _lib().oracle_linear_w8_rows(_p(q), _p(_c(sx, np.float32)), _p(qw), _p(_c(sw, np.float32)), _p(b),
-                                 _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), _p(y))
+    _lib().oracle_linear_w8_rows_act(_p(q), _p(_c(sx, np.float32)), _p(qw), _p(_c(sw, np.float32)), _p(b),
+                                     _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), C.c_int(int(act)), _p(y))
     return y
 
 
-def linear_w4_rows(q, sx, packed, sw4, bias_bits, rows) -> np.ndarray:
+def linear_w4_rows(q, sx, packed, sw4, bias_bits, rows, act: int = 0) -> np.ndarray:
     q = _c(q, np.int8)
     packed = _c(packed, np.uint8)
     rows = _c(rows, np.int64)
@@ -149,8 +149,8 @@ def linear_w4_rows(q, sx, packed, sw4, bias_bits, rows) -> np.ndarray:
     N = packed.shape[0]
     b = None if bias_bits is None else _c(bias_bits, np.uint16)
     y = np.empty((rows.size, N), np.float32)
-    _lib().oracle_linear_w4_rows(_p(q), _p(_c(sx, np.float32)), _p(packed), _p(_c(sw4, np.float32)), _p(b),
-                                 _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), _p(y))
+    _lib().oracle_linear_w4_rows_act(_p(q), _p(_c(sx, np.float32)), _p(packed), _p(_c(sw4, np.float32)), _p(b),
+                                     _p(rows), C.c_int(rows.size), C.c_int(N), C.c_int(K), C.c_int(int(act)), _p(y))
     return y
 
 

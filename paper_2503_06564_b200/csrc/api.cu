@@ -442,7 +442,7 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
 
 static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
                                  const int32_t M[2], const void* bias, void* const Y[2], const int64_t ld[2], bool raw,
-                                 void* stream) {
+                                 void* stream, int act = 0) {
   if (!w || !codes || !M || !Y || !ld || (!raw && !scales)) return TRDQ_ERR_NULL;
   if (M[0] < 0 || M[1] < 0) return TRDQ_ERR_SHAPE;
   const int g = find_group(w->t_bounds, t);
@@ -459,8 +459,8 @@ static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t*
   }
   if (M[0] == 0 && M[1] == 0) return TRDQ_OK;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)) return TRDQ_ERR_ALIGN;
-  if (w->wbits == 8) return launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream));
-  return launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream));
+  if (w->wbits == 8) return launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream), act);
+  return launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream), act);
 }
 
 trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M, const void* bias_bf16,
@@ -471,6 +471,17 @@ trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, c
   void* y[2] = {Y_bf16, nullptr};
   const int64_t l[2] = {ldy, ldy};
   return linear_common(w, t, c, s, m, bias_bf16, y, l, false, stream);
+}
+
+trdq_status trdq_linear_act(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M, const void* bias_bf16,
+                            void* Y_bf16, int64_t ldy, int32_t act, void* stream) {
+  if (act != TRDQ_ACT_NONE && act != TRDQ_ACT_GELU_TANH) return TRDQ_ERR_SHAPE;
+  const int8_t* c[2] = {codes, nullptr};
+  const float* s[2] = {scales, nullptr};
+  const int32_t m[2] = {M, 0};
+  void* y[2] = {Y_bf16, nullptr};
+  const int64_t l[2] = {ldy, ldy};
+  return linear_common(w, t, c, s, m, bias_bf16, y, l, false, stream, act);
 }
 
 trdq_status trdq_linear_cfg(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
@@ -574,12 +585,13 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
     if (op.M > 0 && (!op.X_bf16 || !op.codes || !op.scales || !op.Y_bf16)) return TRDQ_ERR_NULL;
     if (op.ldx % 8 != 0 || op.ldy % 8 != 0 || !aligned16(op.X_bf16) || !aligned16(op.codes) || !aligned16(op.Y_bf16))
       return TRDQ_ERR_ALIGN;
+    if (op.act != TRDQ_ACT_NONE && op.act != TRDQ_ACT_GELU_TANH) return TRDQ_ERR_SHAPE;
   }
   for (int i = 0; i < count; ++i) {
     const trdq_layer_op& op = ops[i];
     trdq_status st = trdq_rotate_quantize(op.rot, t, op.X_bf16, op.ldx, op.M, op.codes, op.scales, stream);
     if (st != TRDQ_OK) return st;
-    st = trdq_linear(op.w, t, op.codes, op.scales, op.M, op.bias_bf16, op.Y_bf16, op.ldy, stream);
+    st = trdq_linear_act(op.w, t, op.codes, op.scales, op.M, op.bias_bf16, op.Y_bf16, op.ldy, op.act, stream);
     if (st != TRDQ_OK) return st;
   }
   return TRDQ_OK;

@@ -22,10 +22,23 @@ __device__ __forceinline__ float dequant_one(int32_t a, float sxm, float swn, fl
   return v;
 }
 
-// 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n], packed to bf16 pairs.
+// GELU in its tanh form, the activation between the two MLP linears of a DiT block:
+//   gelu(x) = 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)) = x exp(2u) / (1 + exp(2u)),   u = sqrt(2/pi) (x + 0.044715 x^3).
+// With e = exp(-|2u|) in (0, 1] the denominator 1 + e stays in [1, 2] on both sides, so nothing overflows and the
+// fast division is in its defined range.  exp through ex2.approx: relative error near 1e-6, far inside a bf16
+// rounding step; results below about 1e-37 in magnitude (x < -10) flush to zero.
+__device__ __forceinline__ float gelu_tanh(float x) {
+  const float k = 1.5957691216057308f;  // 2 sqrt(2/pi)
+  const float t = __fmul_rn(x, __fmaf_rn(__fmul_rn(x, x), 0.044715f * k, k));  // 2u, same sign as x
+  const float e = __expf(-fabsf(t));
+  const float num = t >= 0.0f ? x : __fmul_rn(x, e);
+  return __fdividef(num, __fadd_rn(1.0f, e));
+}
+
+// 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n] (then GELU if act != 0), packed to bf16 pairs.
 // pb4: (sw, bias) of the 32 columns as 16 float4; thr4: 2^-10 * |bias| as 8 float4.
 __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm, const float4* pb4, const float4* thr4,
-                                              uint32_t (&packed)[16]) {
+                                              uint32_t (&packed)[16], int act = 0) {
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
     const float4 p01 = pb4[j / 2], p23 = pb4[j / 2 + 1], th = thr4[j / 4];
@@ -35,6 +48,10 @@ __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm
     float y[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) y[e] = dequant_one(static_cast<int32_t>(r[j + e]), sxm, swv[e], bv[e], tv[e]);
+    if (act) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) y[e] = gelu_tanh(y[e]);
+    }
     const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]);
     const __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2], y[3]);
     packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h0);

@@ -68,6 +68,7 @@ struct alignas(64) GemmParams {
   const int32_t* zp[2];
   const int32_t* colsum;
   int32_t N, K, tiles_n;
+  int32_t act;  // 0: none, 1: GELU (tanh form) on the dequantized value before the bf16 rounding
   // split-K (raw-accumulator mode only): the k-blocks are cut into `splits` ranges of `kb_per_split`; split s
   // writes its partial sums at out + s * split_stride (elements).  splits = 1 is the ordinary GEMM.
   int32_t splits, kb_per_split;
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
           const float4* pb4 = reinterpret_cast<const float4*>(pb + c * 32);
           const float4* thr4 = reinterpret_cast<const float4*>(thr + c * 32);
           uint32_t packed[16];
-          dequant_row32(r, sxm, pb4, thr4, packed);
+          dequant_row32(r, sxm, pb4, thr4, packed, p.act);
           // staging tile: row = lane, 64 bytes per row, 16-byte chunk j stored at j ^ ((lane >> 1) & 3)
           if (lane == 0) bulk_wait_group_read<0>();  // the previous store has finished reading the tile
           __syncwarp();
@@ -334,7 +335,7 @@ int choose_tile_n(int64_t tiles_m, int N, int sms) {
 }  // namespace
 
 static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, int mode,
-                                       const int32_t* const zp[2], cudaStream_t stream) {
+                                       const int32_t* const zp[2], cudaStream_t stream, int act = 0) {
   const bool raw_i32 = mode == 1;
   // Large problems go to the CTA-pair kernel (two SMs per 256-row tile, a third less operand traffic per SM).
   static const int pair_min_rows = [] {
@@ -342,7 +343,7 @@ static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmS
     return e ? atoi(e) : 2048;
   }();
   if (mode == 0 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows) {
-    const trdq_status st = launch_gemm_w8_pair(w, g, seg, bias_bf16, stream);
+    const trdq_status st = launch_gemm_w8_pair(w, g, seg, bias_bf16, stream, act);
     if (st != TRDQ_ERR_SHAPE) return st;
   }
   int dev = 0, sms = 148;
@@ -382,6 +383,7 @@ static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmS
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
+  p.act = act;
   p.splits = 1;
   p.kb_per_split = w->K / kTileKBytes;
   p.split_stride = 0;
@@ -405,8 +407,8 @@ static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmS
 }
 
 trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
-                           cudaStream_t stream) {
-  return launch_gemm_w8_mode(w, g, seg, bias_bf16, raw_i32 ? 1 : 0, nullptr, stream);
+                           cudaStream_t stream, int act) {
+  return launch_gemm_w8_mode(w, g, seg, bias_bf16, raw_i32 ? 1 : 0, nullptr, stream, act);
 }
 
 // Unsigned activation codes with per-row zero points (Eq. 1-3); `w` must carry the column sums of its codes.
@@ -509,6 +511,7 @@ trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegmen
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   GemmParams p;
+  p.act = 0;
   p.sx[0] = p.sx[1] = nullptr;
   p.out[0] = p.out[1] = workspace;
   p.ld[0] = p.ld[1] = w->N;

@@ -57,6 +57,7 @@ struct alignas(64) Gemm2Params {
   const float* sw;
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n;
+  int32_t act;  // 0: none, 1: GELU (tanh form) before the bf16 rounding
   uint32_t* status;
 };
 
@@ -279,7 +280,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
         uint32_t packed[16];
-        dequant_row32(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed);
+        dequant_row32(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed, p.act);
         const uint32_t tile_smem = my_stage + flip * 2048;
         flip ^= 1;
         if (lane == 0) bulk_wait_group_read<1>();  // the store issued two chunks ago has finished reading this tile
@@ -363,7 +364,8 @@ int max_clusters(int dev) {
 }  // namespace
 
 // Returns TRDQ_ERR_SHAPE when the pair kernel does not apply (caller falls back to the single-CTA kernel).
-trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream) {
+trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream,
+                                int act) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   Gemm2Params p;
@@ -408,6 +410,7 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
+  p.act = act;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   const int64_t total = tiles_m * p.tiles_n;

@@ -18,6 +18,7 @@
 // written by TMA stores.  Every wait is bounded.
 #include <cuda_bf16.h>
 
+#include "epilogue.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -56,6 +57,7 @@ struct alignas(64) W4Params {
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n, n_pad;
   int32_t mult_in_smem;  // 1: all K/128 multiplier rows of a tile fit the shared-memory table
+  int32_t act;           // 0: none, 1: GELU (tanh form) before the bf16 rounding
   uint32_t* status;
 };
 
@@ -311,7 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
             const float cm = __fmul_rn(sxm, pb.x);
             float v = __fmaf_rn(sf, cm, pb.y);
             if (fabsf(v) < thr_buf[col]) v = __fmaf_rn(__ll2float_rn(S - __float2ll_rz(sf)), cm, v);  // the part fp32 dropped
-            y[e] = v;
+            y[e] = p.act ? gelu_tanh(v) : v;
           }
           const __nv_bfloat162 h = __floats2bfloat162_rn(y[0], y[1]);
           packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
@@ -373,7 +375,7 @@ cudaError_t launch_w4_multipliers(const float* scales, int32_t N, int32_t groups
   return cudaGetLastError();
 }
 
-trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream) {
+trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream, int act) {
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -399,6 +401,7 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
   p.mult_t = w->groups[g].mult_t;
   p.base = w->groups[g].base;
   p.bias = static_cast<const __nv_bfloat16*>(bias_bf16);
+  p.act = act;
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + kTileNW4 - 1) / kTileNW4;

@@ -85,10 +85,11 @@ struct GemmSegment {
   int64_t ld;
   int32_t M;
 };
+// act: 0 = none, 1 = GELU (tanh form) applied to the dequantized value before the bf16 rounding
 trdq_status launch_gemm_w8(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, bool raw_i32,
-                           cudaStream_t stream);
+                           cudaStream_t stream, int act = 0);
 trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
-                           cudaStream_t stream);
+                           cudaStream_t stream, int act = 0);
 trdq_status launch_gemm_w8_asym(const trdq_weights* w, int g, const GemmSegment seg[2], const int32_t* const zp[2],
                                 const void* bias_bf16, cudaStream_t stream);
 cudaError_t launch_weight_colsum(const int8_t* codes, int32_t N, int32_t K, int32_t* colsum, cudaStream_t stream);
@@ -102,7 +103,7 @@ trdq_status launch_gemm_w8_splitk_static(const trdq_weights* w, int g, const Gem
                                          cudaStream_t stream);
 // gemm_i8_2cta.cu: CTA-pair kernel; TRDQ_ERR_SHAPE means "not applicable here, use the single-CTA kernel"
 trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
-                                cudaStream_t stream);
+                                cudaStream_t stream, int act = 0);
 cudaError_t launch_w4_multipliers(const float* scales, int32_t N, int32_t groups, int32_t n_pad, int32_t* mult_t, float* base,
                                   cudaStream_t stream);
 

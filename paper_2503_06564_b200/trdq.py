@@ -30,7 +30,7 @@ EXPORTS = (
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
     "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
     "trdq_selftest_wait_expiry", "trdq_rotation_create_dense", "trdq_rotate_dense_workspace", "trdq_rotate_dense_quantize",
-    "trdq_greedy_rotation_block",
+    "trdq_greedy_rotation_block", "trdq_linear_act",
 )
 
 
@@ -48,7 +48,7 @@ class RotationSpec(C.Structure):
 class LayerOp(C.Structure):
     _fields_ = [("rot", C.c_void_p), ("w", C.c_void_p), ("X_bf16", C.c_void_p), ("ldx", C.c_int64), ("M", C.c_int32),
                 ("codes", C.c_void_p), ("scales", C.c_void_p), ("bias_bf16", C.c_void_p), ("Y_bf16", C.c_void_p),
-                ("ldy", C.c_int64)]
+                ("ldy", C.c_int64), ("act", C.c_int32)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         l.trdq_weights_export.argtypes = [vp, i32, vp, vp, vp]
         l.trdq_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp]
         l.trdq_linear.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
+        l.trdq_linear_act.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i32, vp]
         l.trdq_linear_cfg.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), vp, C.POINTER(vp),
                                       C.POINTER(i64), vp]
         l.trdq_gemm_i32.argtypes = [vp, i32, vp, i32, vp, i64, vp]
@@ -304,6 +305,21 @@ def trdq_linear(w: Weights, t: int, codes, scales, bias_bf16=None, out=None):
     return out
 
 
+ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def trdq_linear_act(w: Weights, t: int, codes, scales, bias_bf16=None, out=None, act: int = ACT_GELU_TANH):
+    """trdq_linear with the following activation (GELU, tanh form) folded into the epilogue."""
+    import torch
+    M = int(codes.shape[0])
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.bfloat16, device=codes.device)
+    ldy = int(out.stride(0)) if M > 1 else w.N
+    _check(lib().trdq_linear_act(w._h, int(t), _ptr(codes), _ptr(scales), M, _ptr(bias_bf16), _ptr(out), ldy, int(act), _stream()),
+           "trdq_linear_act")
+    return out
+
+
 def trdq_linear_cfg(w: Weights, t: int, codes2, scales2, bias_bf16=None, out2=None):
     """Two row segments (conditional, unconditional) through one launch."""
     import torch
@@ -399,11 +415,11 @@ class LayerList:
         self._ops = []
         self._array = None
 
-    def add(self, rot: Rotation, w: Weights, X_bf16, codes, scales, bias_bf16, Y_bf16) -> None:
+    def add(self, rot: Rotation, w: Weights, X_bf16, codes, scales, bias_bf16, Y_bf16, act: int = 0) -> None:
         M = int(X_bf16.shape[0])
         assert X_bf16.stride(1) == 1 and Y_bf16.stride(1) == 1 and codes.is_contiguous()
         self._ops.append(LayerOp(rot._h, w._h, _ptr(X_bf16), int(X_bf16.stride(0)) if M > 1 else rot.K, M, _ptr(codes),
-                                 _ptr(scales), _ptr(bias_bf16), _ptr(Y_bf16), int(Y_bf16.stride(0)) if M > 1 else w.N))
+                                 _ptr(scales), _ptr(bias_bf16), _ptr(Y_bf16), int(Y_bf16.stride(0)) if M > 1 else w.N, int(act)))
         self._keep.append((rot, w, X_bf16, codes, scales, bias_bf16, Y_bf16))
         self._array = None
 

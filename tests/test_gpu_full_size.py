@@ -106,3 +106,45 @@ def test_run_layers_follows_the_time_step_schedule():
     with pytest.raises(trdq.TrdqError) as e:
         trdq.trdq_run_layers(bad, 0)
     assert e.value.status == 10
+
+
+def test_run_layers_block_with_shared_attention_and_fused_gelu():
+    """One transformer block's four linears as a layer list in which the attention linears see the conditional rows
+    only (the unconditional branch reuses the conditional attention, Sec. 3.3) and the first MLP linear carries its GELU
+    in the epilogue.  Every op must equal the stand-alone calls bit for bit, and the oracle on sampled rows."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(123)
+    hidden, M, M_cond = 1152, 1024, 512
+    bounds = WL.group_bounds(2)
+    shapes = [(hidden, 3 * hidden, M_cond, 0), (hidden, hidden, M_cond, 0), (hidden, 4 * hidden, M, 1), (4 * hidden, hidden, M, 0)]
+    layers = trdq.LayerList()
+    keep = []
+    for K, N, rows, act in shapes:
+        signs = (rng.integers(0, 2, (2, K)) * 2 - 1).astype(np.int8)
+        rot = trdq.Rotation(K, bounds, signs)
+        w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.05)
+        bias_bits = WL.to_bf16_bits(rng.standard_normal(N) * 0.1)
+        w = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), 8)
+        x_bits = WL.to_bf16_bits(rng.standard_normal((rows, K)))
+        x, bias = to_dev_bf16(x_bits), to_dev_bf16(bias_bits)
+        codes = torch.empty((rows, K), dtype=torch.int8, device="cuda")
+        scales = torch.empty((rows,), dtype=torch.float32, device="cuda")
+        y = torch.empty((rows, N), dtype=torch.bfloat16, device="cuda")
+        layers.add(rot, w, x, codes, scales, bias, y, act=act)
+        keep.append((rot, w, x, x_bits, bias, bias_bits, signs, codes, scales, y, act))
+    t = 700
+    trdq.trdq_run_layers(layers, t)
+    g = 1
+    for rot, w, x, x_bits, bias, bias_bits, signs, codes, scales, y, act in keep:
+        c2, s2 = trdq.trdq_rotate_quantize(rot, t, x)
+        y2 = trdq.trdq_linear_act(w, t, c2, s2, bias, act=act)
+        assert torch.equal(c2, codes) and torch.equal(s2, scales) and torch.equal(y2, y)
+        a, _ = O.fused_vectors(signs[g], None)
+        c_ref, s_ref = O.rotate_quantize(x_bits, a)
+        assert np.array_equal(codes.cpu().numpy(), c_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+        wq, sw = w.view_tensors(g)
+        rows = np.arange(0, x.shape[0], 37, dtype=np.int64)
+        y_ref = O.linear_w8_rows(c_ref, s_ref, wq.cpu().numpy(), sw.cpu().numpy(), bias_bits, rows, act=act)
+        check_output(bf16_to_f32_np(y)[rows], y_ref, tiny=2.0 ** -100 if act else 0.0)
+    assert trdq.trdq_device_status() == 0

@@ -321,3 +321,34 @@ def test_an_expired_wait_is_reported_and_the_device_stays_usable():
     y_ref = O.linear_w8_rows(q_ref, sx_ref, qw_ref, sw_ref, bias, np.arange(64))
     check_output(bf16_to_f32_np(y), y_ref, max_ulp=1.0)
     assert trdq.trdq_device_status() == 0
+
+
+@pytest.mark.parametrize("M,K,N,wbits", [(300, 256, 400, 8), (4096, 1152, 4608, 8), (260, 384, 272, 4)])
+def test_linear_with_gelu_epilogue(M, K, N, wbits):
+    """trdq_linear_act: GELU (tanh form) folded into the epilogue, all three GEMM kernels (M >= 2048 takes the CTA-pair one),
+    against the oracle's double evaluation on the same codes; act = 0 must equal trdq_linear bit for bit."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(90 + N)
+    signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs)
+    x = WL.to_bf16_bits(rng.standard_normal((M, K)) * 2.0)
+    w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.06)        # pre-activations of a few units: both GELU tails are hit
+    bias_bits = WL.to_bf16_bits(rng.standard_normal(N) * 0.5)
+    w = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), wbits)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, to_dev_bf16(x))
+    bias = to_dev_bf16(bias_bits)
+    y = trdq.trdq_linear_act(w, 0, codes, scales, bias)
+    wq, sw = w.view_tensors(0)
+    rows = np.unique(np.concatenate([np.arange(0, M, max(1, M // 48)), [M - 1]])).astype(np.int64)
+    fn = O.linear_w8_rows if wbits == 8 else O.linear_w4_rows
+    y_ref = fn(codes.cpu().numpy(), scales.cpu().numpy(), wq.cpu().numpy(), sw.cpu().numpy(), bias_bits, rows, act=1)
+    pre = fn(codes.cpu().numpy(), scales.cpu().numpy(), wq.cpu().numpy(), sw.cpu().numpy(), bias_bits, rows, act=0)
+    assert pre.max() > 3.0 and pre.min() < -3.0
+    check_output(bf16_to_f32_np(y)[rows], y_ref, tiny=2.0 ** -100)   # GELU of x < -8.5 lies below 2^-100
+    plain = trdq.trdq_linear(w, 0, codes, scales, bias)
+    assert torch.equal(trdq.trdq_linear_act(w, 0, codes, scales, bias, act=trdq.ACT_NONE), plain)
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_linear_act(w, 0, codes, scales, bias, act=7)
+    assert e.value.status == 2
+    assert trdq.trdq_device_status() == 0

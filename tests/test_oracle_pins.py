@@ -712,3 +712,43 @@ def test_greedy_block_eq6_structure_and_eq7_choice():
     R1 = C @ Q @ C
     R_one, n_one, _ = O.greedy_block(X, G[:1])
     assert n_one == 1 and np.max(np.abs(R_one - R1)) < 1e-10
+
+
+# --------------------------------------------------------------------------- #
+# activation folded into the epilogue
+# --------------------------------------------------------------------------- #
+def test_linear_with_gelu_is_gelu_of_the_linear():
+    import torch
+    rng = np.random.default_rng(50)
+    M, N, K = 6, 40, 128
+    q = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    qw = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    sx = rng.uniform(2e-3, 8e-3, M).astype(np.float32)       # outputs spread over about [-8, 8]
+    sw = rng.uniform(2e-3, 8e-3, N).astype(np.float32)
+    bias = bf16(rng.standard_normal(N))
+    rows = np.arange(M, dtype=np.int64)
+    acc = q.astype(np.int64) @ qw.astype(np.int64).T
+    pre = acc * sx.astype(np.float64)[:, None] * sw.astype(np.float64)[None, :] + f32_of(bias).astype(np.float64)[None, :]
+    assert np.abs(pre).max() > 4 and np.abs(pre).min() < 0.05
+    got = O.linear_w8_rows(q, sx, qw, sw, bias, rows, act=1).astype(np.float64)
+    # library routine 1: torch's fp64 GELU (tanh form).  It evaluates 0.5 x (1 + tanh u) as printed, which cancels for
+    # x < -4, so it pins the bulk; library routine 2: scipy's logistic function through 0.5 (1 + tanh u) = expit(2u),
+    # accurate on both tails, pins the whole range.
+    ref_torch = torch.nn.functional.gelu(torch.from_numpy(pre), approximate="tanh").numpy()
+    bulk = pre > -4.0
+    assert np.max(np.abs(got - ref_torch)[bulk] / np.maximum(np.abs(ref_torch[bulk]), 1e-30)) < 2.0 ** -22
+    from scipy.special import expit
+    ref = pre * expit(2.0 * np.sqrt(2.0 / np.pi) * (pre + 0.044715 * pre ** 3))
+    assert np.max(np.abs(got - ref) / np.maximum(np.abs(ref), 1e-300)) < 2.0 ** -22
+    assert np.min(pre) < -6.0 and np.min(np.abs(ref)) < 1e-10          # the deep tail is in the sample
+    assert np.array_equal(O.linear_w8_rows(q, sx, qw, sw, bias, rows, act=0), pre.astype(np.float32))
+    # closed-form anchors of the function itself: gelu(0) = 0, gelu(x) -> x for large x, -> 0 for very negative x,
+    # and gelu(x) - gelu(-x) = x
+    one = np.ones((1, 1), np.int8)
+    for x in (0.0, 12.0, -12.0, 0.75):
+        s = np.float32(abs(x)) if x != 0 else np.float32(0.0)
+        y_pos = O.linear_w8_rows(one * (1 if x >= 0 else -1), [s], one, [1.0], None, [0], act=1)[0, 0]
+        y_neg = O.linear_w8_rows(one * (-1 if x >= 0 else 1), [s], one, [1.0], None, [0], act=1)[0, 0]
+        assert abs((y_pos - y_neg) - x) <= 1e-6 * max(1.0, abs(x))
+    assert O.linear_w8_rows(one, [12.0], one, [1.0], None, [0], act=1)[0, 0] == np.float32(12.0)
+    assert abs(O.linear_w8_rows(-one, [12.0], one, [1.0], None, [0], act=1)[0, 0]) < 1e-30
