@@ -660,6 +660,48 @@ int oracle_greedy_block(const double* Xc, int Mc, int steps, const double* gauss
   return best_k;
 }
 
+// ---- normalisation and modulation folded in front of the rotation ------------------------------------------
+// The quantized linears of a DiT block read a LayerNorm output modulated per sample (adaLN):
+//   h[m, k] = (x[m, k] - mean_m) / sqrt(var_m + eps) * (1 + scale[s, k]) + shift[s, k],   s = m / rows_per_sample,
+// mean and (biased) variance over the row's K channels.  Evaluated in double and rounded once to fp32; h then takes the
+// place of the bf16 input of the rotation (oracle_rotate_f32).  scale / shift may be null (zero).  The paper does not
+// discuss normalisation; this backs the fused variant of the online call.
+void oracle_norm_modulate(const uint16_t* x_bf16, int64_t ldx, int M, int K, const uint16_t* shift_bf16, const uint16_t* scale_bf16,
+                          int rows_per_sample, double eps, float* h) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m) {
+    const uint16_t* row = x_bf16 + static_cast<int64_t>(m) * ldx;
+    double mean = 0.0;
+    for (int k = 0; k < K; ++k) mean += static_cast<double>(bf16_to_float(row[k]));
+    mean /= K;
+    double var = 0.0;
+    for (int k = 0; k < K; ++k) {
+      const double d = static_cast<double>(bf16_to_float(row[k])) - mean;
+      var += d * d;
+    }
+    var /= K;
+    const double rstd = 1.0 / std::sqrt(var + eps);
+    const int64_t s = m / rows_per_sample;
+    for (int k = 0; k < K; ++k) {
+      const double sc = scale_bf16 ? static_cast<double>(bf16_to_float(scale_bf16[s * K + k])) : 0.0;
+      const double sh = shift_bf16 ? static_cast<double>(bf16_to_float(shift_bf16[s * K + k])) : 0.0;
+      h[static_cast<int64_t>(m) * K + k] = static_cast<float>((static_cast<double>(bf16_to_float(row[k])) - mean) * rstd * (1.0 + sc) + sh);
+    }
+  }
+}
+
+// The block rotation of oracle_rotate on fp32 rows: u = fl32(h * vec), then the butterfly.
+void oracle_rotate_f32(const float* h, int M, int K, const float* vec, float* v) {
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int c = 0; c < K; c += kBlock) {
+      float u[kBlock];
+      for (int i = 0; i < kBlock; ++i) u[i] = h[static_cast<int64_t>(m) * K + c + i] * vec[c + i];
+      butterfly128(u);
+      for (int i = 0; i < kBlock; ++i) v[static_cast<int64_t>(m) * K + c + i] = u[i];
+    }
+}
+
 int oracle_num_threads() {
   int n = 1;
 #ifdef _OPENMP

@@ -312,3 +312,24 @@ def greedy_block(x_calib, gauss) -> Tuple[np.ndarray, int, np.ndarray]:
     trace = np.empty(steps, np.float64)
     n = int(_lib().oracle_greedy_block(_p(x), C.c_int(x.shape[0]), C.c_int(steps), _p(g), _p(R), _p(trace)))
     return R, n, trace
+
+
+# ---- LayerNorm + modulation in front of the rotation ---------------------------------------------
+
+def norm_modulate(x_bits, shift_bits, scale_bits, rows_per_sample: int, eps: float) -> np.ndarray:
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    sh = None if shift_bits is None else _c(shift_bits, np.uint16)
+    sc = None if scale_bits is None else _c(scale_bits, np.uint16)
+    h = np.empty((M, K), np.float32)
+    _lib().oracle_norm_modulate(_p(x), C.c_int64(K), C.c_int(M), C.c_int(K), _p(sh), _p(sc), C.c_int(int(rows_per_sample)),
+                                C.c_double(float(eps)), _p(h))
+    return h
+
+
+def rotate_f32(h, vec) -> np.ndarray:
+    h = _c(h, np.float32)
+    M, K = h.shape
+    v = np.empty((M, K), np.float32)
+    _lib().oracle_rotate_f32(_p(h), C.c_int(M), C.c_int(K), _p(_c(vec, np.float32)), _p(v))
+    return v

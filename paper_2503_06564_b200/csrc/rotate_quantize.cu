@@ -13,71 +13,11 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "lane_group.cuh"
 #include "ptx.cuh"
 
 namespace trdq {
 namespace {
-
-constexpr int kLanesPerBlock = 8;
-constexpr int kElemsPerLane = 16;
-
-__device__ __forceinline__ void load_scaled16(const uint4* src, const float (&vec)[16], float (&u)[16]) {
-  const uint4 a = __ldg(src);
-  const uint4 b = __ldg(src + 1);
-  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    // bf16 -> fp32 is exact: the 16 bits become the high half of the fp32 pattern
-    const float lo = __uint_as_float(w[i] << 16);
-    const float hi = __uint_as_float(w[i] & 0xFFFF0000u);
-    u[2 * i] = __fmul_rn(lo, vec[2 * i]);
-    u[2 * i + 1] = __fmul_rn(hi, vec[2 * i + 1]);
-  }
-}
-
-// 128-point unnormalised Walsh-Hadamard transform across the 8 lanes of a group, natural
-// (Sylvester) order: stage h maps (a, b) = (u[i], u[i+h]) to (a + b, a - b).
-__device__ __forceinline__ void wht128(float (&u)[16], int lane8) {
-#pragma unroll
-  for (int h = 1; h < 16; h <<= 1) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      if ((i & h) == 0) {
-        const float a = u[i];
-        const float b = u[i + h];
-        u[i] = __fadd_rn(a, b);
-        u[i + h] = __fsub_rn(a, b);
-      }
-    }
-  }
-#pragma unroll
-  for (int mask = 1; mask < 8; mask <<= 1) {
-    const bool upper = (lane8 & mask) != 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float other = __shfl_xor_sync(0xffffffffu, u[i], mask);
-      // lower lane: a + b with a = own; upper lane: a - b with a = other, b = own
-      u[i] = __fadd_rn(other, upper ? -u[i] : u[i]);
-    }
-  }
-}
-
-__device__ __forceinline__ float absmax16(const float (&u)[16]) {
-  float m = 0.0f;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(u[i]));
-  return m;
-}
-
-__device__ __forceinline__ float group_max(float m) {
-  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
-  return m;
-}
-
-// Symmetric quantizer of Eq. 1 with z = 0: q = rne(v * fl(qmax / amax)).
-__device__ __forceinline__ int quantize_one(float v, float inv) { return __float2int_rn(__fmul_rn(v, inv)); }
 
 // MODE 0: int8 per row.  MODE 1: int4 per 128-block, packed.
 // P = blocks handled by one lane group per tile (P > 1 only for very wide rows).

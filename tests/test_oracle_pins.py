@@ -752,3 +752,42 @@ def test_linear_with_gelu_is_gelu_of_the_linear():
         assert abs((y_pos - y_neg) - x) <= 1e-6 * max(1.0, abs(x))
     assert O.linear_w8_rows(one, [12.0], one, [1.0], None, [0], act=1)[0, 0] == np.float32(12.0)
     assert abs(O.linear_w8_rows(-one, [12.0], one, [1.0], None, [0], act=1)[0, 0]) < 1e-30
+
+
+# --------------------------------------------------------------------------- #
+# LayerNorm + modulation folded in front of the rotation
+# --------------------------------------------------------------------------- #
+def test_norm_modulate_is_layer_norm_then_modulation():
+    import torch
+    rng = np.random.default_rng(51)
+    M, K, rps, eps = 12, 256, 4, 1e-6
+    x_bits = bf16(rng.standard_normal((M, K)) * 3.0 + 1.5)
+    shift_bits = bf16(rng.standard_normal((M // rps, K)) * 0.3)
+    scale_bits = bf16(rng.standard_normal((M // rps, K)) * 0.3)
+    x = torch.from_numpy(f32_of(x_bits).astype(np.float64))
+    ln = torch.nn.functional.layer_norm(x, (K,), eps=eps).numpy()                      # library routine, fp64
+    sc = np.repeat(f32_of(scale_bits).astype(np.float64), rps, axis=0)
+    sh = np.repeat(f32_of(shift_bits).astype(np.float64), rps, axis=0)
+    ref = ln * (1.0 + sc) + sh
+    h = O.norm_modulate(x_bits, shift_bits, scale_bits, rps, eps).astype(np.float64)
+    assert np.max(np.abs(h - ref)) <= 2.0 ** -23 * np.max(np.abs(ref))
+    # without modulation it is the plain normalisation: zero mean, unit variance
+    h0 = O.norm_modulate(x_bits, None, None, rps, eps).astype(np.float64)
+    assert np.max(np.abs(h0 - ln)) <= 2.0 ** -22 and np.max(np.abs(h0.mean(axis=1))) < 1e-6
+    assert np.max(np.abs(h0.var(axis=1) - 1.0)) < 1e-5
+    # a constant row has no deviation: the output is the shift; scale = -1 removes the normalised part as well
+    const = bf16(np.full((rps, K), 2.5))
+    assert np.array_equal(O.norm_modulate(const, shift_bits[:1], scale_bits[:1], rps, eps), np.repeat(f32_of(shift_bits[:1]), rps, axis=0))
+    minus_one = bf16(np.full((1, K), -1.0))
+    assert np.array_equal(O.norm_modulate(x_bits[:rps], shift_bits[:1], minus_one, rps, eps), np.repeat(f32_of(shift_bits[:1]), rps, axis=0))
+    # the sample index: rows of the second sample use the second modulation row
+    swapped = O.norm_modulate(x_bits[rps:2 * rps], shift_bits[1:2], scale_bits[1:2], rps, eps)
+    assert np.array_equal(swapped, O.norm_modulate(x_bits, shift_bits, scale_bits, rps, eps)[rps:2 * rps])
+
+
+def test_rotate_f32_equals_rotate_on_bf16_values():
+    rng = np.random.default_rng(52)
+    x_bits = bf16(rng.standard_normal((5, 384)))
+    signs = (rng.integers(0, 2, 384) * 2 - 1).astype(np.int8)
+    a, _ = O.fused_vectors(signs, rng.uniform(0.5, 2.0, 384).astype(np.float32))
+    assert np.array_equal(O.rotate_f32(f32_of(x_bits), a), O.rotate(x_bits, a))
