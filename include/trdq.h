@@ -212,6 +212,20 @@ trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const
 trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
                              int32_t M, const void* bias_bf16, void* Y_bf16, int64_t ldy, void* stream);
 
+/* trdq_rotate_quantize with the producer of its input folded in: the quantized linears of a transformer block read a
+ * LayerNorm output modulated per sample (adaLN),
+ *   h[m,k] = (X[m,k] - mean_m) / sqrt(var_m + eps) * (1 + scale[s,k]) + shift[s,k],   s = m / rows_per_sample,
+ * mean and biased variance over the K channels of row m.  h is formed in fp32 in registers (never stored, not rounded to
+ * bf16) and takes the place of X in Eq. 10's G_t: v = (h o Delta_t) R_t, then the per-token quantizer, codes and scales as
+ * in trdq_rotate_quantize.  shift_bf16 / scale_bf16: dev bf16 [ceil(M / rows_per_sample), K], 16-byte aligned, or NULL (zero).
+ * Single Hadamard rotation only (TRDQ_ERR_MISMATCH for the full transform or dense blocks); K <= 8192; eps >= 0.
+ * The reductions run in a fixed order, so equal inputs give equal codes.  The row statistics are fp32 sums; against an
+ * evaluation in double h agrees to about 2^-18 relative to its terms, which moves a code only at a rounding boundary.
+ * The paper does not discuss normalisation; this is a fusion on the boundary of its layer. */
+trdq_status trdq_norm_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M,
+                                      const void* shift_bf16, const void* scale_bf16, int32_t rows_per_sample, float eps, int8_t* codes,
+                                      float* scales, void* stream);
+
 /* trdq_linear with the activation that follows the layer folded into its epilogue, so that the activation costs no
  * pass over memory of its own (the first MLP linear of a transformer block is followed by GELU, and its output is what
  * the next trdq_rotate_quantize reads):

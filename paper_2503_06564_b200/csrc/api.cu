@@ -440,6 +440,25 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
+trdq_status trdq_norm_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M,
+                                      const void* shift_bf16, const void* scale_bf16, int32_t rows_per_sample, float eps, int8_t* codes,
+                                      float* scales, void* stream) {
+  if (!rot) return TRDQ_ERR_NULL;
+  if (rot->dense || rot->perm) return TRDQ_ERR_MISMATCH;
+  if (M < 0 || rot->K > 8192 || rows_per_sample <= 0 || !(eps >= 0.0f) || !std::isfinite(eps)) return TRDQ_ERR_SHAPE;
+  const int g = find_group(rot->t_bounds, t);
+  if (g < 0) return TRDQ_ERR_TIMESTEP;
+  if (M == 0) return TRDQ_OK;
+  if (!X_bf16 || !codes || !scales) return TRDQ_ERR_NULL;
+  if (ldx < rot->K) return TRDQ_ERR_SHAPE;
+  if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u) ||
+      (shift_bf16 && !aligned16(shift_bf16)) || (scale_bf16 && !aligned16(scale_bf16)))
+    return TRDQ_ERR_ALIGN;
+  const cudaError_t e = launch_norm_rotate_quantize(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, shift_bf16,
+                                                    scale_bf16, rows_per_sample, eps, codes, scales, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+}
+
 static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
                                  const int32_t M[2], const void* bias, void* const Y[2], const int64_t ld[2], bool raw,
                                  void* stream, int act = 0) {

@@ -69,6 +69,11 @@ bool rotate_quantize_prefers_tma(int32_t M, int32_t K);
 trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
                                        float* scales, cudaStream_t stream);
 
+// norm_rotate_quantize.cu: LayerNorm + per-sample modulation in front of the rotation (K <= 8192)
+cudaError_t launch_norm_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, const void* shift_bf16,
+                                        const void* scale_bf16, int32_t rows_per_sample, float eps, int8_t* codes, float* scales,
+                                        cudaStream_t stream);
+
 // rotate_dense.cu: dense block rotation on the tensor cores + per-token quantizer (two passes over X)
 uint64_t rotate_dense_workspace_bytes(int32_t M, int32_t K);
 trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const void* x_bf16, int64_t ldx, int32_t M, int8_t* codes,

@@ -69,4 +69,58 @@ __device__ __forceinline__ float group_max(float m) {
 // Symmetric quantizer of Eq. 1 with z = 0: q = rne(v * fl(qmax / amax)).
 __device__ __forceinline__ int quantize_one(float v, float inv) { return __float2int_rn(__fmul_rn(v, inv)); }
 
+// ---- four lanes per 128-block, fp32 pairs (see the layout description in rotate_quantize.cu) ----
+constexpr int kFastLanes = 4;
+constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23
+
+__device__ __forceinline__ float2 shfl_xor2(float2 v, int mask) {
+  return make_float2(__shfl_xor_sync(0xffffffffu, v.x, mask), __shfl_xor_sync(0xffffffffu, v.y, mask));
+}
+
+__device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
+  const uint32_t lo = __byte_perm(__float_as_uint(a.x), __float_as_uint(a.y), 0x0040);
+  const uint32_t hi = __byte_perm(__float_as_uint(b.x), __float_as_uint(b.y), 0x0040);
+  return __byte_perm(lo, hi, 0x5410);
+}
+
+// 128-point transform of one block spread over four lanes (16 fp32 pairs per lane, layout as described above).
+__device__ __forceinline__ void wht128_lanes4(float2 (&v)[16], int lane4) {
+  // h = 1: inside a pair
+#pragma unroll
+  for (int p = 0; p < 16; ++p) v[p] = make_float2(__fadd_rn(v[p].x, v[p].y), __fsub_rn(v[p].x, v[p].y));
+  // h = 2, 4: pair index bits 0, 1
+#pragma unroll
+  for (int hb = 1; hb <= 2; hb <<= 1) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if ((p & hb) == 0) {
+        const float2 a = v[p], c2 = v[p + hb];
+        v[p] = __fadd2_rn(a, c2);
+        v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+      }
+    }
+  }
+  // h = 8, 16: lanes l ^ 1, l ^ 2; upper lane computes other - own, lower lane own + other
+#pragma unroll
+  for (int mask = 1; mask <= 2; mask <<= 1) {
+    const float sgn = (lane4 & mask) ? -1.0f : 1.0f;
+    const float2 s2 = make_float2(sgn, sgn);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) v[p] = __ffma2_rn(v[p], s2, shfl_xor2(v[p], mask));
+  }
+  // h = 32, 64: pair index bits 2, 3 (the chunk of the lane)
+#pragma unroll
+  for (int hb = 4; hb <= 8; hb <<= 1) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if ((p & hb) == 0) {
+        const float2 a = v[p], c2 = v[p + hb];
+        v[p] = __fadd2_rn(a, c2);
+        v[p + hb] = __ffma2_rn(c2, make_float2(-1.0f, -1.0f), a);  // a - c, one rounding
+      }
+    }
+  }
+
+}
+
 }  // namespace trdq

@@ -3,6 +3,7 @@
     python -m paper_2503_06564_b200.microbench rq   --M 65536 --K 1152
     python -m paper_2503_06564_b200.microbench gemm --M 16384 --K 1152 --N 4608
     python -m paper_2503_06564_b200.microbench rqd  --M 16384 --K 1152      (dense block rotation, Eq. 6-8)
+    python -m paper_2503_06564_b200.microbench nrq  --M 16384 --K 1152      (LayerNorm + modulation folded in front)
 
 Also the small, self-ending command to put under a profiler (few launches, a few hundred MB).
 Buffers are rotated through `--sets` distinct copies so that consecutive launches do not find
@@ -20,7 +21,7 @@ def main():
     import torch
     from paper_2503_06564_b200 import build, trdq
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["rq", "rqd", "gemm"])
+    ap.add_argument("kernel", choices=["rq", "rqd", "nrq", "gemm"])
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--K", type=int, default=1152)
     ap.add_argument("--N", type=int, default=4608)
@@ -53,6 +54,15 @@ def main():
         def run(i):
             s = i % args.sets
             trdq.trdq_rotate_dense_quantize(drot, 0, xs[s], codes[s], scales[s], ws)
+        work, unit = M * (3.0 * K + 4.0) / 1e9, "GB/s"
+    elif args.kernel == "nrq":
+        rps = 256
+        shift = (torch.randn(((M + rps - 1) // rps, K), device="cuda") * 0.2).to(torch.bfloat16)
+        scale = (torch.randn(((M + rps - 1) // rps, K), device="cuda") * 0.2).to(torch.bfloat16)
+
+        def run(i):
+            s = i % args.sets
+            trdq.trdq_norm_rotate_quantize(rot, 0, xs[s], shift, scale, rps, 1e-6, codes[s], scales[s])
         work, unit = M * (3.0 * K + 4.0) / 1e9, "GB/s"
     elif args.kernel == "rq":
         def run(i):

@@ -30,7 +30,7 @@ EXPORTS = (
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
     "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
     "trdq_selftest_wait_expiry", "trdq_rotation_create_dense", "trdq_rotate_dense_workspace", "trdq_rotate_dense_quantize",
-    "trdq_greedy_rotation_block", "trdq_linear_act",
+    "trdq_greedy_rotation_block", "trdq_linear_act", "trdq_norm_rotate_quantize",
 )
 
 
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         l.trdq_weights_export.argtypes = [vp, i32, vp, vp, vp]
         l.trdq_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp]
         l.trdq_linear.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
+        l.trdq_norm_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, i32, C.c_float, vp, vp, vp]
         l.trdq_linear_act.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i32, vp]
         l.trdq_linear_cfg.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), vp, C.POINTER(vp),
                                       C.POINTER(i64), vp]
@@ -253,6 +254,25 @@ def trdq_rotate_quantize(rot: Rotation, t: int, X_bf16, codes=None, scales=None)
     ldx = int(X_bf16.stride(0)) if M > 1 else rot.K
     _check(lib().trdq_rotate_quantize(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(codes), _ptr(scales), _stream()),
            "trdq_rotate_quantize")
+    return codes, scales
+
+
+def trdq_norm_rotate_quantize(rot: Rotation, t: int, X_bf16, shift_bf16=None, scale_bf16=None, rows_per_sample: Optional[int] = None,
+                              eps: float = 1e-6, codes=None, scales=None):
+    """LayerNorm + per-sample modulation + rotation + per-token quantizer in one kernel."""
+    import torch
+    assert X_bf16.is_cuda and X_bf16.dim() == 2 and X_bf16.element_size() == 2 and X_bf16.stride(1) == 1
+    M = int(X_bf16.shape[0])
+    if rows_per_sample is None:
+        rows_per_sample = max(M, 1)
+    if codes is None:
+        codes = torch.empty((M, rot.K), dtype=torch.int8, device=X_bf16.device)
+    if scales is None:
+        scales = torch.empty((M,), dtype=torch.float32, device=X_bf16.device)
+    ldx = int(X_bf16.stride(0)) if M > 1 else rot.K
+    _check(lib().trdq_norm_rotate_quantize(rot._h, int(t), _ptr(X_bf16), ldx, M, _ptr(shift_bf16), _ptr(scale_bf16),
+                                           int(rows_per_sample), float(eps), _ptr(codes), _ptr(scales), _stream()),
+           "trdq_norm_rotate_quantize")
     return codes, scales
 
 

@@ -11,7 +11,7 @@ import pytest
 
 from oracle import trdq_oracle as O
 from paper_2503_06564_b200 import workloads as WL
-from tests.util import bf16_to_f32_np, check_output, to_dev_bf16
+from tests.util import bf16_to_f32_np, check_codes_with_tolerance, check_output, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -46,27 +46,10 @@ def check_dense_codes(codes, scales, x_bits, stored_bits):
     """Compares GPU codes / scales with the oracle under the accumulation tolerance; returns the number of differing codes."""
     K = x_bits.shape[1]
     v = O.rotate_dense(x_bits, stored_bits)
-    c_ref, s_ref = O.quantize_rows(v)
     x = np.abs(WL.bf16_bits_to_f32(x_bits).astype(np.float64))
     S = np.abs(WL.bf16_bits_to_f32(stored_bits).astype(np.float64))
     mass = np.concatenate([x[:, 128 * b:128 * (b + 1)] @ S[b] for b in range(K // 128)], axis=1)   # sum_i |x_i S_ij|
-    tol_v = ACC_TOL * mass
-    amax = np.abs(v).max(axis=1).astype(np.float64)
-    tol_amax = tol_v.max(axis=1)
-    assert np.all(np.abs(scales.astype(np.float64) - s_ref) <= tol_amax / 127.0 * 1.001 + 2.0 ** -23 * s_ref)
-    assert not np.any(codes == -128)
-    diff = codes.astype(np.int32) - c_ref
-    bad = diff != 0
-    if bad.any():
-        assert np.abs(diff).max() <= 1
-        safe = np.where(amax > 0, amax, 1.0)
-        inv = 127.0 / safe
-        u = v.astype(np.float64) * inv[:, None]
-        du = inv[:, None] * tol_v + 127.0 * (tol_amax / safe)[:, None] + 2.0 ** -15
-        dist = np.abs(u - np.floor(u) - 0.5)
-        assert np.all(dist[bad] <= du[bad]), "a differing code is not at a rounding boundary"
-        assert bad.sum() <= 2e-3 * codes.size, f"{bad.sum()} of {codes.size} codes differ"
-    return int(bad.sum())
+    return check_codes_with_tolerance(codes, scales, v, ACC_TOL * mass)
 
 
 @pytest.mark.parametrize("M,K,G", [(300, 1152, 2), (129, 384, 1), (1, 128, 1), (1000, 4608, 1), (128, 256, 3), (77, 2048, 1)])

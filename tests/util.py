@@ -54,3 +54,27 @@ def check_output(y_gpu: np.ndarray, y_ref: np.ndarray, max_ulp: float = 2.0, rel
     assert l2 <= rel_l2, f"relative L2 error {l2:.3e} > {rel_l2}"
     assert ulps.max() <= max_ulp, f"max error {ulps.max():.3f} bf16 ulp at {np.unravel_index(ulps.argmax(), ulps.shape)}"
     return float(l2), float(ulps.max())
+
+
+def check_codes_with_tolerance(codes: np.ndarray, scales: np.ndarray, v_ref: np.ndarray, tol_v: np.ndarray, max_fraction: float = 2e-3):
+    """Codes and scales of a path whose pre-quantization values v agree with the oracle's only up to tol_v (elementwise,
+    absolute): scales may differ by the tolerance at the row maximum (over 127), a code may differ by one step and only
+    where the oracle's value before rounding lies within the propagated tolerance of a .5 boundary.  Returns the count."""
+    from oracle import trdq_oracle as O
+    c_ref, s_ref = O.quantize_rows(v_ref)
+    amax = np.abs(v_ref).max(axis=1).astype(np.float64)
+    tol_amax = np.broadcast_to(tol_v, v_ref.shape).max(axis=1)
+    assert np.all(np.abs(scales.astype(np.float64) - s_ref) <= tol_amax / 127.0 * 1.001 + 2.0 ** -23 * s_ref), "scales out of tolerance"
+    assert not np.any(codes == -128)
+    diff = codes.astype(np.int32) - c_ref
+    bad = diff != 0
+    if bad.any():
+        assert np.abs(diff).max() <= 1, "codes differ by more than one step"
+        safe = np.where(amax > 0, amax, 1.0)
+        inv = 127.0 / safe
+        u = v_ref.astype(np.float64) * inv[:, None]
+        du = inv[:, None] * tol_v + 127.0 * (tol_amax / safe)[:, None] + 2.0 ** -15
+        dist = np.abs(u - np.floor(u) - 0.5)
+        assert np.all(dist[bad] <= du[bad]), "a differing code is not at a rounding boundary"
+        assert bad.sum() <= max_fraction * codes.size, f"{bad.sum()} of {codes.size} codes differ"
+    return int(bad.sum())
