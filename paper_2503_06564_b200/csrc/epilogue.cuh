@@ -35,10 +35,11 @@ __device__ __forceinline__ float gelu_tanh(float x) {
   return __fdividef(num, __fadd_rn(1.0f, e));
 }
 
-// 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n] (then GELU if act != 0), packed to bf16 pairs.
+// 32 consecutive columns of one output row: y = acc * sx * sw[n] + bias[n] (then GELU if ACT), packed to bf16 pairs.
 // pb4: (sw, bias) of the 32 columns as 16 float4; thr4: 2^-10 * |bias| as 8 float4.
+template <bool ACT = false>
 __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm, const float4* pb4, const float4* thr4,
-                                              uint32_t (&packed)[16], int act = 0) {
+                                              uint32_t (&packed)[16]) {
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
     const float4 p01 = pb4[j / 2], p23 = pb4[j / 2 + 1], th = thr4[j / 4];
@@ -48,7 +49,7 @@ __device__ __forceinline__ void dequant_row32(const uint32_t (&r)[32], float sxm
     float y[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) y[e] = dequant_one(static_cast<int32_t>(r[j + e]), sxm, swv[e], bv[e], tv[e]);
-    if (act) {
+    if (ACT) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) y[e] = gelu_tanh(y[e]);
     }

@@ -68,7 +68,6 @@ struct alignas(64) GemmParams {
   const int32_t* zp[2];
   const int32_t* colsum;
   int32_t N, K, tiles_n;
-  int32_t act;  // 0: none, 1: GELU (tanh form) on the dequantized value before the bf16 rounding
   // split-K (raw-accumulator mode only): the k-blocks are cut into `splits` ranges of `kb_per_split`; split s
   // writes its partial sums at out + s * split_stride (elements).  splits = 1 is the ordinary GEMM.
   int32_t splits, kb_per_split;
@@ -96,6 +95,7 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile, i
 
 // MODE 0: bf16 dequantizing epilogue.  MODE 1: raw int32 accumulators.
 // MODE 2: unsigned activation codes with zero points (Eq. 1-3): acc - z[m] * colsum[n], then the epilogue of mode 0.
+// MODE 3: mode 0 with GELU (tanh form) applied to the dequantized value before the bf16 rounding.
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<BN>;
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
           const float4* pb4 = reinterpret_cast<const float4*>(pb + c * 32);
           const float4* thr4 = reinterpret_cast<const float4*>(thr + c * 32);
           uint32_t packed[16];
-          dequant_row32(r, sxm, pb4, thr4, packed, p.act);
+          dequant_row32<MODE == 3>(r, sxm, pb4, thr4, packed);
           // staging tile: row = lane, 64 bytes per row, 16-byte chunk j stored at j ^ ((lane >> 1) & 3)
           if (lane == 0) bulk_wait_group_read<0>();  // the previous store has finished reading the tile
           __syncwarp();
@@ -383,7 +383,6 @@ static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmS
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
-  p.act = act;
   p.splits = 1;
   p.kb_per_split = w->K / kTileKBytes;
   p.split_stride = 0;
@@ -400,6 +399,8 @@ static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmS
     e = bn == 128 ? launch_one<128, 1>(p, grid, stream) : bn == 192 ? launch_one<192, 1>(p, grid, stream) : launch_one<256, 1>(p, grid, stream);
   } else if (mode == 2) {
     e = bn == 128 ? launch_one<128, 2>(p, grid, stream) : bn == 192 ? launch_one<192, 2>(p, grid, stream) : launch_one<256, 2>(p, grid, stream);
+  } else if (act) {
+    e = bn == 128 ? launch_one<128, 3>(p, grid, stream) : bn == 192 ? launch_one<192, 3>(p, grid, stream) : launch_one<256, 3>(p, grid, stream);
   } else {
     e = bn == 128 ? launch_one<128, 0>(p, grid, stream) : bn == 192 ? launch_one<192, 0>(p, grid, stream) : launch_one<256, 0>(p, grid, stream);
   }
@@ -511,7 +512,6 @@ trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegmen
   if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   GemmParams p;
-  p.act = 0;
   p.sx[0] = p.sx[1] = nullptr;
   p.out[0] = p.out[1] = workspace;
   p.ld[0] = p.ld[1] = w->N;

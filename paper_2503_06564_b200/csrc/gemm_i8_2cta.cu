@@ -57,7 +57,6 @@ struct alignas(64) Gemm2Params {
   const float* sw;
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n;
-  int32_t act;  // 0: none, 1: GELU (tanh form) before the bf16 rounding
   uint32_t* status;
 };
 
@@ -132,7 +131,8 @@ __host__ __device__ constexpr uint32_t umma_idesc_s8_pair(int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
 }
 
-template <int BN>
+// ACT: GELU (tanh form) on the dequantized value before the bf16 rounding.
+template <int BN, bool ACT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8a8_pair_kernel(const __grid_constant__ Gemm2Params p) {
   using C = Cfg2<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -280,7 +280,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
         uint32_t packed[16];
-        dequant_row32(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed, p.act);
+        dequant_row32<ACT>(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed);
         const uint32_t tile_smem = my_stage + flip * 2048;
         flip ^= 1;
         if (lane == 0) bulk_wait_group_read<1>();  // the store issued two chunks ago has finished reading this tile
@@ -318,7 +318,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
   }
 }
 
-template <int BN>
+template <int BN, bool ACT>
 cudaError_t launch_pair(const Gemm2Params& p, int clusters, cudaStream_t stream) {
   using C = Cfg2<BN>;
   cudaLaunchConfig_t cfg = {};
@@ -331,7 +331,7 @@ cudaError_t launch_pair(const Gemm2Params& p, int clusters, cudaStream_t stream)
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_w8a8_pair_kernel<BN>, p);
+  return cudaLaunchKernelEx(&cfg, gemm_w8a8_pair_kernel<BN, ACT>, p);
 }
 
 // Clusters of two CTAs that can be resident at once (at most SMs / 2; fewer if a GPC has an odd SM count).
@@ -341,7 +341,8 @@ int max_clusters(int dev) {
   if (dev < 0 || dev >= 16) return 0;
   if (cached[dev] == 0) {
     using C = Cfg2<BN>;
-    if (cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) {
+    if (cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) {
       cudaGetLastError();
       cached[dev] = -1;
       return 0;
@@ -351,7 +352,7 @@ int max_clusters(int dev) {
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_w8a8_pair_kernel<BN>, &cfg) != cudaSuccess || n <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_w8a8_pair_kernel<BN, false>, &cfg) != cudaSuccess || n <= 0) {
       cudaGetLastError();
       cached[dev] = -1;
       return 0;
@@ -410,12 +411,15 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
-  p.act = act;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   const int64_t total = tiles_m * p.tiles_n;
   const int clusters = static_cast<int>(total < clusters_of[best] ? total : clusters_of[best]);
-  const cudaError_t e = bn == 128 ? launch_pair<128>(p, clusters, stream) : bn == 192 ? launch_pair<192>(p, clusters, stream) : launch_pair<256>(p, clusters, stream);
+  cudaError_t e;
+  if (act)
+    e = bn == 128 ? launch_pair<128, true>(p, clusters, stream) : bn == 192 ? launch_pair<192, true>(p, clusters, stream) : launch_pair<256, true>(p, clusters, stream);
+  else
+    e = bn == 128 ? launch_pair<128, false>(p, clusters, stream) : bn == 192 ? launch_pair<192, false>(p, clusters, stream) : launch_pair<256, false>(p, clusters, stream);
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 

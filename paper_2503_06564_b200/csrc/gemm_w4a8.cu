@@ -57,7 +57,6 @@ struct alignas(64) W4Params {
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n, n_pad;
   int32_t mult_in_smem;  // 1: all K/128 multiplier rows of a tile fit the shared-memory table
-  int32_t act;           // 0: none, 1: GELU (tanh form) before the bf16 rounding
   uint32_t* status;
 };
 
@@ -76,6 +75,8 @@ __device__ __forceinline__ TileCoord tile_coord(const W4Params& p, int tile) {
   return c;
 }
 
+// ACT: GELU (tanh form) on the dequantized value before the bf16 rounding.
+template <bool ACT>
 __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_constant__ W4Params p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -313,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w4a8_kernel(const __grid_con
             const float cm = __fmul_rn(sxm, pb.x);
             float v = __fmaf_rn(sf, cm, pb.y);
             if (fabsf(v) < thr_buf[col]) v = __fmaf_rn(__ll2float_rn(S - __float2ll_rz(sf)), cm, v);  // the part fp32 dropped
-            y[e] = p.act ? gelu_tanh(v) : v;
+            y[e] = ACT ? gelu_tanh(v) : v;
           }
           const __nv_bfloat162 h = __floats2bfloat162_rn(y[0], y[1]);
           packed[j / 2] = *reinterpret_cast<const uint32_t*>(&h);
@@ -401,7 +402,6 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
   p.mult_t = w->groups[g].mult_t;
   p.base = w->groups[g].base;
   p.bias = static_cast<const __nv_bfloat16*>(bias_bf16);
-  p.act = act;
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + kTileNW4 - 1) / kTileNW4;
@@ -415,12 +415,15 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
   const int grid = static_cast<int>(total < sms ? total : sms);
   static bool configured[16] = {};
   if (dev >= 0 && dev < 16 && !configured[dev]) {
-    if (cudaFuncSetAttribute(gemm_w4a8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kFixedSmemBytes + kMaxSmemGroups * kTileNW4 * 4) != cudaSuccess)
+    const int max_smem = kFixedSmemBytes + kMaxSmemGroups * kTileNW4 * 4;
+    if (cudaFuncSetAttribute(gemm_w4a8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
       return TRDQ_ERR_CUDA;
     configured[dev] = true;
   }
-  return launch_overlapped(gemm_w4a8_kernel, dim3(grid), dim3(kThreads), smem_bytes, stream, p) == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  const cudaError_t e = act ? launch_overlapped(gemm_w4a8_kernel<true>, dim3(grid), dim3(kThreads), smem_bytes, stream, p)
+                            : launch_overlapped(gemm_w4a8_kernel<false>, dim3(grid), dim3(kThreads), smem_bytes, stream, p);
+  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }
 
 }  // namespace trdq
