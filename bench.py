@@ -29,8 +29,9 @@ METRIC = "rotated_w8a8_linear_tops"
 UNIT = "TOPS"
 # DRAM traffic per unit of algorithmic work, from the Nsight Compute captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch); None once a kernel has changed since its capture.
-GEMM_PAIR_DRAM_BYTES_PER_OP = 130.5e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
+GEMM_PAIR_DRAM_BYTES_PER_OP = 129.6e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
 RQ_TMA_DRAM_BYTES_PER_ALG_BYTE = 191.7 / 226.6      # rotate_quantize_tma_kernel, M = 65536, K = 1152
+RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE = 20.8 / 31.1       # rotate_quantize_rows_kernel, M = 9000, K = 1152
 INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -377,7 +378,17 @@ def run_ours(args, wl: WL.Workload):
     bf16_peak = peaks["bf16_tflops_sustained"] if in_long_step else peaks["bf16_tflops"]
     int8_peak = bf16_peak * INT8_OVER_BF16
     gemm_kernel = "gemm_w4a8_kernel" if wl.wbits == 4 else ("gemm_w8a8_pair_kernel" if wl.M >= 2048 else "gemm_w8a8_kernel")
-    rq_kernel = "rotate_quantize_tma_kernel" if wl.M >= 9472 else "rotate_quantize_rows_kernel"
+    # which rotate + quantize kernel the library picks per layer (rows of <= 36 blocks and >= 6 rounds of one tile per SM
+    # go to the TMA-staged kernel), and the kernel that moves most of the step's bytes
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rq_bytes = {"rotate_quantize_tma_kernel": 0.0, "rotate_quantize_rows_kernel": 0.0}
+    for layer in wl.layers + wl.extra_layers:
+        m, nb = (layer.M or wl.M), layer.K // 128
+        r = (288 // nb) // 8 * 8 if nb <= 36 else 0
+        tma = r > 0 and (m + r - 1) // r >= 6 * sms
+        rq_bytes["rotate_quantize_tma_kernel" if tma else "rotate_quantize_rows_kernel"] += m * (3.0 * layer.K + 4.0)
+    rq_kernel = max(rq_bytes, key=rq_bytes.get)
+    rq_traffic_ratio = RQ_TMA_DRAM_BYTES_PER_ALG_BYTE if rq_kernel == "rotate_quantize_tma_kernel" else RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE
     gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
     rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
     line = {
@@ -398,8 +409,8 @@ def run_ours(args, wl: WL.Workload):
                      "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
         "roofline_rotate_quantize": {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
-                                     "traffic": RQ_TMA_DRAM_BYTES_PER_ALG_BYTE * step_rq_bytes(wl) / n_ops,
-                                     "traffic_note": "bytes per launch: TMA-kernel capture at M=65536,K=1152 scaled by algorithmic bytes",
+                                     "traffic": rq_traffic_ratio * step_rq_bytes(wl) / n_ops,
+                                     "traffic_note": "bytes per launch: capture of this kernel (TMA: M=65536,K=1152; rows: M=9000,K=1152) scaled by algorithmic bytes",
                                      "peak_source": peaks["_source"]},
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},

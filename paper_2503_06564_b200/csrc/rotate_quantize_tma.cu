@@ -222,15 +222,17 @@ int rotate_quantize_tma_rows(int32_t K) {
   return rows >= 8 ? rows : 0;
 }
 
-// The one-thread-per-block kernel keeps a whole tile of R rows in the registers of one CTA, so it needs
-// at least two tiles per SM to overlap one tile's arithmetic with the next one's loads; below that the
-// lane-group kernel, which spreads the same rows over twice as many smaller CTAs, finishes sooner.
+// The one-thread-per-block kernel keeps a whole tile of R rows in the registers of one CTA (one CTA per SM), so its
+// time comes in rounds of one tile per SM, plus the fill of its ring; the lane-group kernel spreads the same rows over
+// twice as many smaller CTAs with finer tiles.  Measured crossover (K = 1024 .. 4608): with fewer than about six
+// rounds the lane-group kernel finishes sooner (by 6 - 14 % at 2.6 - 5.2 rounds), from 6.9 rounds on this one wins
+// (by 5 - 23 %).
 bool rotate_quantize_prefers_tma(int32_t M, int32_t K) {
   const int R = rotate_quantize_tma_rows(K);
   if (R == 0) return false;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  return static_cast<int64_t>(M) >= 2ll * sms * R;
+  return (static_cast<int64_t>(M) + R - 1) / R >= 6ll * sms;
 }
 
 trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,

@@ -38,9 +38,10 @@ def _x(M, K, seed, outliers=True):
     (100, 640, 2, True),        # 5 blocks: 56 rows per tile, the last warp is partly idle, ragged last tile
     (9, 4736, 1, True),         # 37 blocks: too wide for one thread per block, lane-group kernel
     (600, 1152, 1, False),
-    (9500, 1152, 1, True),      # enough rows for the one-thread-per-block TMA kernel: 297 tiles, ring wraps, ragged tail
-    (2400, 4608, 1, False),     # same kernel, 36 blocks, 8 rows per tile
-    (19000, 640, 2, True),      # same kernel, 5 blocks: 56 rows per tile, partly idle last warp
+    (9500, 1152, 1, True),      # 297 tiles of 32 rows: still the lane-group kernel (fewer than six rounds of one tile per SM)
+    (28500, 1152, 1, True),     # enough rows for the one-thread-per-block TMA kernel: 891 tiles, ring wraps, ragged tail
+    (7200, 4608, 1, False),     # same kernel, 36 blocks, 8 rows per tile
+    (50000, 640, 2, True),      # same kernel, 5 blocks: 56 rows per tile, partly idle last warp
 ])
 def test_rotate_quantize_matches_oracle(M, K, G, smooth):
     from paper_2503_06564_b200 import trdq
