@@ -362,12 +362,38 @@ def run_ours(args, wl: WL.Workload):
     h2d = sum(h.numel() * h.element_size() for h in host_x)
     d2h = sum(h.numel() * h.element_size() for h in host_y)
 
+    # Copies and kernels are pipelined layer by layer over three streams (PCIe carries both directions at once): layer i's
+    # kernels wait for its input copy, its output copy waits for its kernels; across steps a buffer is not overwritten before
+    # its reader of the step before has finished.
+    s_main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(n_ops)]
+    ev_done = [torch.cuda.Event() for _ in range(n_ops)]
+    ev_out = [torch.cuda.Event() for _ in range(n_ops)]
+    first_e2e = [True]
+
     def e2e_step(i):
-        for hx, k in zip(host_x, layers._keep):
-            k[2].copy_(hx, non_blocking=True)
-        step(i)
-        for hy, k in zip(host_y, layers._keep):
-            hy.copy_(k[6], non_blocking=True)
+        t = int(ts[i % len(ts)])
+        s_in.wait_stream(s_main)        # buffers written before this step (warm-up, the step before) are complete
+        s_out.wait_stream(s_main)
+        for j, (hx, hy, k) in enumerate(zip(host_x, host_y, layers._keep)):
+            with torch.cuda.stream(s_in):
+                if not first_e2e[0]:
+                    s_in.wait_event(ev_done[j])       # the step before has read X_j
+                k[2].copy_(hx, non_blocking=True)
+                ev_in[j].record(s_in)
+            s_main.wait_event(ev_in[j])
+            if not first_e2e[0]:
+                s_main.wait_event(ev_out[j])          # the step before has copied Y_j out
+            trdq.trdq_run_layers(layers, t, first=j, count=1)
+            ev_done[j].record(s_main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[j])
+                hy.copy_(k[6], non_blocking=True)
+                ev_out[j].record(s_out)
+        first_e2e[0] = False
+        s_main.wait_stream(s_in)
+        s_main.wait_stream(s_out)       # the step's results are on the host when the timed region ends
 
     e2e_step(0)
     ms_e2e = time_region(e2e_step, e2e_steps) / e2e_steps
