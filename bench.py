@@ -29,7 +29,7 @@ METRIC = "rotated_w8a8_linear_tops"
 UNIT = "TOPS"
 # DRAM traffic per unit of algorithmic work, from the Nsight Compute captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch); None once a kernel has changed since its capture.
-GEMM_PAIR_DRAM_BYTES_PER_OP = 129.6e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
+GEMM_PAIR_DRAM_BYTES_PER_OP = 123.3e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
 RQ_TMA_DRAM_BYTES_PER_ALG_BYTE = 191.7 / 226.6      # rotate_quantize_tma_kernel, M = 65536, K = 1152
 RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE = 20.8 / 31.1       # rotate_quantize_rows_kernel, M = 9000, K = 1152
 INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)

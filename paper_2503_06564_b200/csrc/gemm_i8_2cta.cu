@@ -13,8 +13,8 @@
 //   empty[s]   in each CTA: tcgen05.commit multicast to both CTAs when the MMAs reading stage s are done
 //   tfull[a]   in each CTA: tcgen05.commit multicast when accumulator a is complete
 //   tempty[a]  in the LEADER: the epilogue warps of both CTAs arrive (16 arrivals)
-// The epilogue is the single-CTA kernel's (one row per thread, eight warps per CTA), with two staging
-// tiles per warp so that a TMA store overlaps the next chunk's arithmetic.  No TMA multicast is used.
+// The epilogue is the single-CTA kernel's (one row per thread, eight warps per CTA), but stores two 32-column chunks
+// at a time (a 32 x 64 bf16 tile per TMA store: whole 128-byte lines).  No TMA multicast is used.
 #include <cuda_bf16.h>
 
 #include "epilogue.cuh"
@@ -40,7 +40,7 @@ struct Cfg2 {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kParamBytes = 2 * BN * 12;
   static constexpr int kBarrierBytes = 256;
-  static constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 2 * 2048;  // two 32 x 32 bf16 tiles per warp
+  static constexpr int kOutStageBytes = (kEpilogueThreads / 32) * 4096;  // one 32 x 64 bf16 tile per warp
   static constexpr int kStages = (kSmemBudget - 1024 - kOutStageBytes - kParamBytes - kBarrierBytes) / kStageBytes;
   static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kParamBytes + kBarrierBytes;
   static_assert(kStages >= 3 && kStages <= 10, "stage count out of range");
@@ -50,7 +50,8 @@ struct Cfg2 {
 struct alignas(64) Gemm2Params {
   CUtensorMap tmap_a[2];    // codes of each segment, box 128 B x 128 rows
   CUtensorMap tmap_b;       // weights, box 128 B x BN/2 rows
-  CUtensorMap tmap_out[2];  // bf16 output, box 32 x 32, 64-byte swizzle
+  CUtensorMap tmap_out[2];     // bf16 output, box 64 x 32, 128-byte swizzle: two 32-column chunks per store
+  CUtensorMap tmap_out32[2];   // box 32 x 32, 64-byte swizzle: the odd chunk of BN = 192
   const float* sx[2];
   int32_t M[2];
   int32_t pair_tiles_m[2];  // 256-row tiles per segment
@@ -182,6 +183,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
     prefetch_tensormap(&p.tmap_b);
     prefetch_tensormap(&p.tmap_out[0]);
     prefetch_tensormap(&p.tmap_out[1]);
+    if ((BN / 64) % 2) {
+      prefetch_tensormap(&p.tmap_out32[0]);
+      prefetch_tensormap(&p.tmap_out32[1]);
+    }
   }
   griddep_launch_dependents();
   griddep_wait();
@@ -258,7 +263,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
     BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
     int acc = 0;
     uint32_t acc_phase = 0;
-    uint32_t flip = 0;
     for (int tile = cluster_id; tile < total_tiles; tile += num_clusters) {
       const TileCoord tc = pair_tile_coord(p, tile, BN);
       const int m0 = tc.m0 + rank * kTileM;
@@ -273,26 +277,52 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
       __syncwarp();
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccStride;
+      // two 32-column chunks per store: a 32 x 64 bf16 tile (128-byte rows, 128-byte swizzle), full lines on the way out
 #pragma unroll 1
-      for (int cc = 0; cc < kChunksPerWarp; ++cc) {
+      for (int cc = 0; cc + 1 < kChunksPerWarp; cc += 2) {
         const int c = half * kChunksPerWarp + cc;
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+          uint32_t r[32];
+          tmem_ld_32x32(t_row + (c + h2) * 32, r);
+          tmem_wait_ld();
+          uint32_t packed[16];
+          dequant_row32<ACT>(r, sxm, reinterpret_cast<const float4*>(pb + (c + h2) * 32), reinterpret_cast<const float4*>(thr + (c + h2) * 32),
+                             packed);
+          if (h2 == 0) {
+            if (lane == 0) bulk_wait_group_read<0>();  // the previous store has finished reading the tile
+            __syncwarp();
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            st_shared_v4(my_stage + lane * 128 + (((4 * h2 + v) ^ (lane & 7)) << 4), packed[4 * v], packed[4 * v + 1], packed[4 * v + 2],
+                         packed[4 * v + 3]);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&p.tmap_out[tc.seg], tc.n0 + c * 32, m0 + q * 32, my_stage);  // rows >= M and columns >= N are clipped
+          bulk_commit_group();
+        }
+      }
+      if (kChunksPerWarp % 2) {
+        // the odd chunk (BN = 192): a 32 x 32 tile, 64-byte rows, chunk v stored at v ^ ((lane >> 1) & 3)
+        const int c = half * kChunksPerWarp + kChunksPerWarp - 1;
         uint32_t r[32];
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
         uint32_t packed[16];
         dequant_row32<ACT>(r, sxm, reinterpret_cast<const float4*>(pb + c * 32), reinterpret_cast<const float4*>(thr + c * 32), packed);
-        const uint32_t tile_smem = my_stage + flip * 2048;
-        flip ^= 1;
-        if (lane == 0) bulk_wait_group_read<1>();  // the store issued two chunks ago has finished reading this tile
+        if (lane == 0) bulk_wait_group_read<0>();
         __syncwarp();
 #pragma unroll
         for (int v = 0; v < 4; ++v)
-          st_shared_v4(tile_smem + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4), packed[4 * v], packed[4 * v + 1], packed[4 * v + 2],
+          st_shared_v4(my_stage + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4), packed[4 * v], packed[4 * v + 1], packed[4 * v + 2],
                        packed[4 * v + 3]);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d(&p.tmap_out[tc.seg], tc.n0 + c * 32, m0 + q * 32, tile_smem);  // rows >= M and columns >= N are clipped
+          tma_store_2d(&p.tmap_out32[tc.seg], tc.n0 + c * 32, m0 + q * 32, my_stage);
           bulk_commit_group();
         }
       }
@@ -402,6 +432,9 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
                                           static_cast<uint64_t>(w->K), kTileKBytes, kTileM);
     if (st != TRDQ_OK) return st;
     st = encode_tmap_2d(&p.tmap_out[s], src.out, 2, static_cast<uint64_t>(w->N), static_cast<uint64_t>(src.M),
+                        static_cast<uint64_t>(src.ld) * 2, 64, 32, 128);
+    if (st != TRDQ_OK) return st;
+    st = encode_tmap_2d(&p.tmap_out32[s], src.out, 2, static_cast<uint64_t>(w->N), static_cast<uint64_t>(src.M),
                         static_cast<uint64_t>(src.ld) * 2, 32, 32, 64);
     if (st != TRDQ_OK) return st;
   }
