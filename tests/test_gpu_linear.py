@@ -352,3 +352,44 @@ def test_linear_with_gelu_epilogue(M, K, N, wbits):
         trdq.trdq_linear_act(w, 0, codes, scales, bias, act=7)
     assert e.value.status == 2
     assert trdq.trdq_device_status() == 0
+
+
+@pytest.mark.parametrize("wbits", [8, 4])
+def test_maximum_k(wbits):
+    """K = 131072, the largest row the interface accepts (the bound that keeps |sum q * qw| <= K * 127^2 below 2^31):
+    1024 blocks per row through the wide-row rotate kernel, 1024 k-blocks through the GEMM.  With every activation and
+    weight code at +-127 in a worst-case row the accumulator reaches K * 127^2 = 2 114 060 288 exactly."""
+    from paper_2503_06564_b200 import trdq
+    K, M, N = 131072, 5, 32
+    rng = np.random.default_rng(77)
+    signs = np.ones((1, K), np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs, np.full((1, K), 2.0 ** 3.5, np.float32))     # fused vector exactly +1
+    x = rng.standard_normal((M, K))
+    w = rng.standard_normal((N, K)) * 0.05
+    # one token and one output channel made of a single spike per block: the transform of a spike is flat, so every
+    # rotated value of that row is +-amax and every code +-127
+    spike = np.zeros(K)
+    spike[::128] = 3.0
+    x[0] = spike
+    w[0] = spike * 0.01
+    x_bits, w_bits = WL.to_bf16_bits(x), WL.to_bf16_bits(w)
+    wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), wbits)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, to_dev_bf16(x_bits))
+    act, wv = O.fused_vectors(signs[0], np.full(K, 2.0 ** 3.5, np.float32))
+    q_ref, sx_ref = O.rotate_quantize(x_bits, act)
+    assert np.array_equal(codes.cpu().numpy(), q_ref) and np.array_equal(scales.cpu().numpy(), sx_ref)
+    assert np.all(np.abs(q_ref[0]) == 127)                                  # the flat row
+    y = trdq.trdq_linear(wts, 0, codes, scales, None)
+    rows = np.arange(M)
+    if wbits == 8:
+        qw_ref, sw_ref = O.prepare_w8(w_bits, wv)
+        acc = trdq.trdq_gemm_i32(wts, 0, codes).cpu().numpy()
+        acc_ref = O.gemm_i32(q_ref, qw_ref)
+        assert np.array_equal(acc, acc_ref)
+        assert abs(int(acc_ref[0, 0])) == K * 127 * 127                     # the int32 bound is reached, not exceeded
+        y_ref = O.linear_w8_rows(q_ref, sx_ref, qw_ref, sw_ref, None, rows)
+    else:
+        pk_ref, sw4_ref = O.prepare_w4(w_bits, wv)
+        y_ref = O.linear_w4_rows(q_ref, sx_ref, pk_ref, sw4_ref, None, rows)
+    check_output(bf16_to_f32_np(y), y_ref)
+    assert trdq.trdq_device_status() == 0
