@@ -127,6 +127,24 @@ trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_byt
 trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint32_t box_cols, uint64_t rows,
                               uint64_t row_stride_bytes, uint32_t boxes, uint32_t box_rows);
 
+// Tile height for the row kernels that run two CTAs per SM over tiles of whole rows: the CTAs work through the tiles
+// in rounds, a round costs about (rows + 2) row-times, and slightly smaller tiles can fill the last round
+// (M = 4096, K = 1152: 7 rows give 586 tiles = 1.98 rounds of 296 CTAs, 8 rows give 1.73 rounds that cost 2).
+inline int rows_per_tile_by_rounds(int32_t M, int rows_max, int sms) {
+  int rows = rows_max;
+  long best_cost = -1;
+  for (int cand = rows_max; cand >= (rows_max + 1) / 2; --cand) {
+    const long tiles = (M + cand - 1) / cand;
+    const long rounds = (tiles + 2 * sms - 1) / (2 * sms);
+    const long cost = rounds * (cand + 2);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      rows = cand;
+    }
+  }
+  return rows;
+}
+
 // Launches `kernel` so that its prologue may overlap the tail of the previous kernel in the stream
 // (the kernel itself orders its memory accesses with griddep_wait()).
 template <typename... KArgs, typename... Args>

@@ -185,12 +185,12 @@ cudaError_t launch_norm_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t
                                         cudaStream_t stream) {
   const int nb = K / TRDQ_BLOCK;
   if (nb > 64) return cudaErrorInvalidValue;  // one row must fit a CTA: K <= 8192
-  int rows = std::max(1, std::min(32, 72 / nb));  // about 72 lane groups (288 threads) per CTA
-  const int threads = (rows * nb * kFastLanes + 31) / 32 * 32;
-  const size_t smem = (static_cast<size_t>(K) + 4u * rows * nb) * sizeof(float);
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int rows = rows_per_tile_by_rounds(M, std::max(1, std::min(32, 72 / nb)), sms);  // at most about 72 lane groups (288 threads) per CTA
+  const int threads = (rows * nb * kFastLanes + 31) / 32 * 32;
+  const size_t smem = (static_cast<size_t>(K) + 4u * rows * nb) * sizeof(float);
   const int num_tiles = (M + rows - 1) / rows;
   const int grid = std::min(num_tiles, sms * 2);
   return launch_overlapped(norm_rotate_quantize_rows_kernel<2>, dim3(grid), dim3(threads), smem, stream,

@@ -40,17 +40,17 @@ constexpr int kBarrierBytes = 256;
 // pass 0: ring of (X tile, S_b) pairs
 constexpr int kStages0 = 3;
 constexpr int kSmemBytes0 = 1024 + kStages0 * 2 * kTileBytes + kBarrierBytes;
-// pass 1: resident S_b, ring of X tiles, per drain warp two staging tiles of 32 rows x 64 codes
+// pass 1: resident S_b, ring of X tiles, one staging tile per drain warp
 constexpr int kStages1 = 4;
 constexpr int kDrainWarps1 = 8;
-constexpr int kOutStageBytes = kDrainWarps1 * 2 * 2048;
+constexpr int kOutStageBytes = kDrainWarps1 * 4096;  // per drain warp one staging tile of 32 rows x 128 codes
 constexpr int kSmemBytes1 = 1024 + kTileBytes + kStages1 * kTileBytes + kOutStageBytes + kBarrierBytes;
 constexpr float kRoundMagic = 12582912.0f;          // 1.5 * 2^23: adding it leaves rne(u) in the low mantissa bits
 
 struct alignas(64) DenseParams {
   CUtensorMap tmap_x;      // bf16 [M, K] (row stride ldx), box 64 columns x 128 rows, 128-byte swizzle
   CUtensorMap tmap_s;      // bf16 [G * K/128 * 128, 128]: S_b transposed (row j = output channel), same box
-  CUtensorMap tmap_codes;  // int8 [M, K], box 64 x 32, 64-byte swizzle
+  CUtensorMap tmap_codes;  // int8 [M, K], box 128 x 32, 128-byte swizzle
   float* amax;             // [splits][M]: max of |v| over the row's blocks of each split
   float* scales;           // [M]
   int32_t M, K;
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) rotate_dense_quantize_kernel(cons
     }
     for (int a = 0; a < kAccSlots; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, kDrainWarps1);
+      mbar_init(bar_tempty + 8 * a, kDrainWarps1 / 2);  // the four warps that drain this tile
     }
     mbar_init(bar_s, 1);
     fence_mbar_init();
@@ -307,12 +307,12 @@ __global__ void __launch_bounds__(kThreads, 1) rotate_dense_quantize_kernel(cons
     }
   } else if (warp >= 4) {
     const int ew = warp - 4;
-    const int q = ew & 3;      // = warp % 4: the lane quarter of tensor memory this warp may read
-    const int half = ew >> 2;  // which 64 of the 128 columns
-    const uint32_t my_stage = out_stage_base + ew * 4096;
+    const int q = ew & 3;        // = warp % 4: the lane quarter of tensor memory this warp may read
+    const int parity = ew >> 2;  // warps 4-7 drain this CTA's even tiles, warps 8-11 the odd ones: 32 rows x all 128 columns each,
+                                 // so that a store writes whole 128-byte lines of the code matrix
+    const uint32_t tile_smem = out_stage_base + ew * 4096;
     BoundedWaiter w(p.status, kStatusTimeoutEpilogue);
-    Pipe acc;
-    // the row maxima of the next tile are fetched while the current one is drained (raw values are kept in
+    // the row maxima of this warp's next tile are fetched while the current one is drained (raw values are kept in
     // registers and only combined one iteration later, so that the loads never stall this warp)
     float part[kMaxSplits];
     auto fetch = [&](int it) {
@@ -320,25 +320,24 @@ __global__ void __launch_bounds__(kThreads, 1) rotate_dense_quantize_kernel(cons
 #pragma unroll
       for (int s = 0; s < kMaxSplits; ++s) part[s] = (s < p.splits && row < p.M) ? __ldg(p.amax + static_cast<size_t>(s) * p.M + row) : 0.0f;
     };
-    if (my_tiles > 0) fetch(0);
-    for (int it = 0; it < my_tiles; ++it) {
+    if (parity < my_tiles) fetch(parity);
+    for (int it = parity; it < my_tiles; it += 2) {
+      const int acc_idx = it & (kAccSlots - 1);
+      const uint32_t acc_phase = (it / kAccSlots) & 1;
       const int row0 = tile_row0(it);
       const int row = row0 + q * 32 + lane;
       float amax = part[0];
 #pragma unroll
       for (int s = 1; s < kMaxSplits; ++s) amax = fmaxf(amax, part[s]);
-      if (it + 1 < my_tiles) fetch(it + 1);
-      if (row < p.M && b == 0 && half == 0) p.scales[row] = __fdiv_rn(amax, 127.0f);
+      if (it + 2 < my_tiles) fetch(it + 2);
+      if (row < p.M && b == 0) p.scales[row] = __fdiv_rn(amax, 127.0f);
       const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-      w.wait(bar_tfull + 8 * acc.idx, acc.phase);
+      w.wait(bar_tfull + 8 * acc_idx, acc_phase);
       __syncwarp();
       tc_fence_after();
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc.idx * kAccCols + half * 64;
-      const uint32_t tile_smem = my_stage + (it & 1) * 2048;
-      if (lane == 0) bulk_wait_group_read<1>();  // the store issued two tiles ago has finished reading this buffer
-      __syncwarp();
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc_idx * kAccCols;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
         tmem_ld_32x32(t_row + c * 32, r);
         tmem_wait_ld();
@@ -350,19 +349,22 @@ __global__ void __launch_bounds__(kThreads, 1) rotate_dense_quantize_kernel(cons
           for (int e = 0; e < 4; ++e) by[e] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r[4 * j + e]), inv), kRoundMagic));
           wds[j] = __byte_perm(__byte_perm(by[0], by[1], 0x0040), __byte_perm(by[2], by[3], 0x0040), 0x5410);
         }
-        // staging tile: row = lane, 64 bytes per row, 16-byte chunk v stored at v ^ ((lane >> 1) & 3)
-        st_shared_v4(tile_smem + lane * 64 + (((2 * c) ^ ((lane >> 1) & 3)) << 4), wds[0], wds[1], wds[2], wds[3]);
-        st_shared_v4(tile_smem + lane * 64 + (((2 * c + 1) ^ ((lane >> 1) & 3)) << 4), wds[4], wds[5], wds[6], wds[7]);
+        if (c == 0) {
+          if (lane == 0) bulk_wait_group_read<0>();  // this warp's previous store has finished reading the buffer
+          __syncwarp();
+        }
+        // staging tile: row = lane, 128 bytes per row, 16-byte chunk v stored at v ^ (lane & 7)
+        st_shared_v4(tile_smem + lane * 128 + (((2 * c) ^ (lane & 7)) << 4), wds[0], wds[1], wds[2], wds[3]);
+        st_shared_v4(tile_smem + lane * 128 + (((2 * c + 1) ^ (lane & 7)) << 4), wds[4], wds[5], wds[6], wds[7]);
       }
       tc_fence_before();
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(bar_tempty + 8 * acc.idx);
-        tma_store_2d(&p.tmap_codes, b * TRDQ_BLOCK + half * 64, row0 + q * 32, tile_smem);  // rows >= M are clipped
+        mbar_arrive(bar_tempty + 8 * acc_idx);
+        tma_store_2d(&p.tmap_codes, b * TRDQ_BLOCK, row0 + q * 32, tile_smem);  // rows >= M are clipped
         bulk_commit_group();
       }
-      acc.advance(kAccSlots);
     }
     if (lane == 0) bulk_wait_group_read<0>();
     w.settle();
@@ -485,7 +487,7 @@ trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const 
   trdq_status st = encode_tmap_2d(&p.tmap_x, x_bf16, 2, K, M, static_cast<uint64_t>(ldx) * 2, 64, kRows, 128);
   if (st != TRDQ_OK) return st;
   p.tmap_s = rot->tmap_dense;
-  st = encode_tmap_2d(&p.tmap_codes, codes, 1, K, M, K, 64, 32, 64);
+  st = encode_tmap_2d(&p.tmap_codes, codes, 1, K, M, K, 128, 32, 128);
   if (st != TRDQ_OK) return st;
   p.amax = workspace;
   p.scales = scales;

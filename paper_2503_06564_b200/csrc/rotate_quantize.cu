@@ -12,6 +12,8 @@
 // combined through a shared-memory atomic max on the (non-negative) float bit patterns.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "internal.h"
 #include "lane_group.cuh"
 #include "ptx.cuh"
@@ -569,19 +571,7 @@ cudaError_t launch_rows_fast(const void* x, int64_t ldx, int32_t M, int32_t K, c
   int rows_max = 72 / nb;  // about 72 lane groups (288 threads) per CTA
   if (rows_max < 1) rows_max = 1;
   if (rows_max > 32) rows_max = 32;
-  // Two CTAs per SM work through the tiles in rounds; a round costs about (rows + 2) row-times.  Slightly smaller tiles
-  // can fill the last round (M = 4096, K = 1152: 7 rows give 586 tiles = 1.98 rounds, 8 rows give 1.73 rounds that cost 2).
-  int rows = rows_max;
-  long best_cost = -1;
-  for (int cand = rows_max; cand >= (rows_max + 1) / 2; --cand) {
-    const long tiles = (M + cand - 1) / cand;
-    const long rounds = (tiles + 2 * sms - 1) / (2 * sms);
-    const long cost = rounds * (cand + 2);
-    if (best_cost < 0 || cost < best_cost) {
-      best_cost = cost;
-      rows = cand;
-    }
-  }
+  const int rows = rows_per_tile_by_rounds(M, rows_max, sms);
   int threads = rows * nb * kFastLanes;
   threads = (threads + 31) / 32 * 32;
   const int num_tiles = (M + rows - 1) / rows;
@@ -633,14 +623,12 @@ cudaError_t launch_rotate_quantize_asym(const void* x_bf16, int64_t ldx, int32_t
   if (M == 0) return cudaSuccess;
   const int nb = K / TRDQ_BLOCK;
   if (nb > 80) return cudaErrorInvalidValue;
-  int rows = 72 / nb;
-  if (rows < 1) rows = 1;
-  if (rows > 32) rows = 32;
-  int threads = rows * nb * kFastLanes;
-  threads = (threads + 31) / 32 * 32;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int rows = rows_per_tile_by_rounds(M, std::max(1, std::min(32, 72 / nb)), sms);
+  int threads = rows * nb * kFastLanes;
+  threads = (threads + 31) / 32 * 32;
   const int num_tiles = (M + rows - 1) / rows;
   return launch_overlapped(rotate_quantize_rows_asym_kernel<2>, dim3(min(num_tiles, sms * 2)), dim3(threads),
                            static_cast<size_t>(K) * sizeof(float), stream, static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec, codes,
