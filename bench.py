@@ -139,7 +139,7 @@ def make_device_x(wl: WL.Workload, M: int, K: int, gen):
     return x.to(torch.bfloat16)
 
 
-def build_device_workload(wl: WL.Workload, seed: int, blocks: int):
+def build_device_workload(wl: WL.Workload, seed: int, blocks: int, rotation: str = "hadamard"):
     """Distinct weights, activations and outputs for every linear of every block, so that one step
     streams a working set far larger than L2."""
     import torch
@@ -149,6 +149,7 @@ def build_device_workload(wl: WL.Workload, seed: int, blocks: int):
     layers = trdq.LayerList()
     alphas = WL.group_alphas(wl.num_groups)
     rng = np.random.default_rng(seed)
+    dense_blocks = {}
     for b in range(blocks):
         for layer in wl.layers + wl.extra_layers:
             M = layer.M or wl.M
@@ -158,13 +159,26 @@ def build_device_workload(wl: WL.Workload, seed: int, blocks: int):
             ax = x.abs().amax(dim=0).double().clamp_min(1e-5).cpu().numpy()
             aw = w.abs().amax(dim=0).double().clamp_min(1e-5).cpu().numpy()
             smooth = np.stack([1.0 / (ax ** a / aw ** (1.0 - a)) for a in alphas]).astype(np.float32)
-            signs = (rng.integers(0, 2, (wl.num_groups, layer.K)) * 2 - 1).astype(np.int8)
-            rot = trdq.Rotation(layer.K, wl.t_bounds, signs, smooth)
+            ws = None
+            if rotation == "dense":
+                # Eq. 6-8: dense 128 x 128 orthogonal blocks per group (random ones stand in for calibrated products; one set
+                # per C_in is reused by every layer of that width, each layer still folds in its own smoothing vector)
+                if layer.K not in dense_blocks:
+                    blk = np.empty((wl.num_groups, layer.K // 128, 128, 128), np.float32)
+                    for g in range(wl.num_groups):
+                        for j in range(layer.K // 128):
+                            blk[g, j] = np.linalg.qr(rng.standard_normal((128, 128)))[0]
+                    dense_blocks[layer.K] = blk
+                rot = trdq.DenseRotation(layer.K, wl.t_bounds, dense_blocks[layer.K], smooth)
+                ws = torch.empty((trdq.trdq_rotate_dense_workspace(rot, M),), dtype=torch.uint8, device="cuda")
+            else:
+                signs = (rng.integers(0, 2, (wl.num_groups, layer.K)) * 2 - 1).astype(np.int8)
+                rot = trdq.Rotation(layer.K, wl.t_bounds, signs, smooth)
             wts = trdq.trdq_prepare_weights(rot, w, wl.wbits)
             codes = torch.empty((M, layer.K), dtype=torch.int8, device="cuda")
             scales = torch.empty((M,), dtype=torch.float32, device="cuda")
             y = torch.empty((M, layer.N), dtype=torch.bfloat16, device="cuda")
-            layers.add(rot, wts, x, codes, scales, bias, y)
+            layers.add(rot, wts, x, codes, scales, bias, y, workspace=ws)
             del w
     torch.cuda.synchronize()
     return layers
@@ -192,8 +206,10 @@ def kernel_pass_ms(layers, wl, which: str, reps: int):
     keep = layers._keep
 
     def issue():
-        for rot, w, x, codes, scales, bias, y in keep:
-            if which == "rq":
+        for (rot, w, x, codes, scales, bias, y), ws in zip(keep, layers._extra):
+            if which == "rq" and ws is not None:
+                trdq.trdq_rotate_dense_quantize(rot, t, x, codes, scales, ws)
+            elif which == "rq":
                 trdq.trdq_rotate_quantize(rot, t, x, codes, scales)
             else:
                 trdq.trdq_linear(w, t, codes, scales, bias, y)
@@ -322,7 +338,7 @@ def run_ours(args, wl: WL.Workload):
     trdq.lib()                                   # fails loudly if the CUDA library is missing
 
     # weak scaling: every rank runs the whole workload on its own batch (rows are independent; no collective)
-    layers = build_device_workload(wl, seed=1234 + rank, blocks=wl.blocks)
+    layers = build_device_workload(wl, seed=1234 + rank, blocks=wl.blocks, rotation=args.rotation)
     ts = wl.timesteps()
     n_ops = len(layers)
 
@@ -415,6 +431,9 @@ def run_ours(args, wl: WL.Workload):
         rq_bytes["rotate_quantize_tma_kernel" if tma else "rotate_quantize_rows_kernel"] += m * (3.0 * layer.K + 4.0)
     rq_kernel = max(rq_bytes, key=rq_bytes.get)
     rq_traffic_ratio = RQ_TMA_DRAM_BYTES_PER_ALG_BYTE if rq_kernel == "rotate_quantize_tma_kernel" else RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE
+    dense = args.rotation == "dense"
+    if dense:
+        rq_kernel, rq_traffic_ratio = "rotate_dense_amax_kernel+rotate_dense_quantize_kernel", None
     gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
     rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
     line = {
@@ -423,6 +442,7 @@ def run_ours(args, wl: WL.Workload):
         "dtype": "int8" if wl.wbits == 8 else "int8xint4", "data": "synthetic",
         "config": {"workload": wl.name, "M": wl.M, "blocks": wl.blocks, "linears_per_step": n_ops, "groups": wl.num_groups,
                    "sampling_steps": wl.steps, "wbits": wl.wbits, "parallelism": f"replicas x{world} (rows independent)",
+                   "rotation": args.rotation,
                    "l2": "inputs larger than L2: every linear has its own X, codes, Y and weights"},
         "us_per_dit_step": ms_per_step * 1e3,
         "rotate_quantize_gbs": rq_gbs,
@@ -435,16 +455,16 @@ def run_ours(args, wl: WL.Workload):
                      "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
         "roofline_rotate_quantize": {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
-                                     "traffic": rq_traffic_ratio * step_rq_bytes(wl) / n_ops,
+                                     "traffic": None if rq_traffic_ratio is None else rq_traffic_ratio * step_rq_bytes(wl) / n_ops,
                                      "traffic_note": "bytes per launch: capture of this kernel (TMA: M=65536,K=1152; rows: M=9000,K=1152) scaled by algorithmic bytes",
                                      "peak_source": peaks["_source"]},
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},
-        "gpu_launches": 2 * n_ops * args.steps,
+        "gpu_launches": (3 if dense else 2) * n_ops * args.steps,
         "clocks": clocks,
     }
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not dense:
             line["cpu_baseline"] = cpu_baseline(wl)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -460,6 +480,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into the workload list (1 = DiT-XL/2 256px, M = 4096)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rotation", default="hadamard", choices=["hadamard", "dense"],
+                    help="hadamard: the headline path; dense: dense 128 x 128 blocks on the tensor cores (Eq. 6-8), no CPU baseline")
     args = ap.parse_args()
     wl = WL.WORKLOADS[args.workload]
     if args.impl == "reference":

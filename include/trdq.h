@@ -249,7 +249,8 @@ trdq_status trdq_linear_act(const trdq_weights* w, int32_t t, const int8_t* code
  *   wr[n, 128 b + j] = fl32( sum_i (S_b^-1)[j][i] * W[n, 128 b + i] )      sums in double, i ascending.
  * TRDQ_ERR_GROUP: bounds not ascending, a non-positive smooth value, a non-finite product or a singular block.
  * The object is accepted by trdq_prepare_weights, trdq_group_of, trdq_rotate_dense_quantize and
- * trdq_rotation_destroy; the Hadamard entry points (trdq_rotate_quantize, _asym, trdq_run_layers) return TRDQ_ERR_MISMATCH. */
+ * trdq_rotation_destroy, and by trdq_run_layers through the op's workspace; the Hadamard entry points (trdq_rotate_quantize,
+ * _asym, trdq_norm_rotate_quantize) return TRDQ_ERR_MISMATCH. */
 trdq_status trdq_rotation_create_dense(int32_t K, int32_t num_groups, const int32_t* t_bounds, const float* blocks, const float* smooth,
                                        trdq_rotation** out);
 
@@ -291,12 +292,15 @@ typedef struct trdq_layer_op {
   void* Y_bf16;             /* dev [M, ldy] */
   int64_t ldy;
   int32_t act;              /* TRDQ_ACT_NONE or TRDQ_ACT_GELU_TANH: activation folded into this layer's epilogue */
+  void* workspace;          /* only for a rot made by trdq_rotation_create_dense: scratch of trdq_rotate_dense_quantize */
+  uint64_t workspace_bytes; /* at least what trdq_rotate_dense_workspace reports for M; ignored otherwise */
 } trdq_layer_op;
 
 /* Runs `count` layer ops in order for time-step t on `stream`: the group switch of the sampling
  * loop (Sec. 3.2: every layer selects its parameter set by the current time-step) without one
  * host round trip per kernel.  Validates every op before launching anything.  TRDQ_ERR_MISMATCH
- * if an op's rot and w disagree in K or in their time-step bounds.
+ * if an op's rot and w disagree in K or in their time-step bounds.  An op whose rot holds dense blocks runs
+ * trdq_rotate_dense_quantize with the op's workspace (TRDQ_ERR_NULL / TRDQ_ERR_NOMEM if it is missing or too small).
  * Every op has its own row count M, so a block whose unconditional branch reuses the conditional
  * attention (attention sharing, Sec. 3.3) lists its attention linears with the conditional rows only
  * and its MLP linears with all rows; nothing is computed for the skipped rows. */

@@ -598,7 +598,11 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
   for (int i = 0; i < count; ++i) {
     const trdq_layer_op& op = ops[i];
     if (!op.rot || !op.w) return TRDQ_ERR_NULL;
-    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds || op.rot->dense) return TRDQ_ERR_MISMATCH;
+    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds) return TRDQ_ERR_MISMATCH;
+    if (op.rot->dense && op.M > 0) {
+      if (!op.workspace) return TRDQ_ERR_NULL;
+      if (op.workspace_bytes < rotate_dense_workspace_bytes(op.M, op.rot->K)) return TRDQ_ERR_NOMEM;
+    }
     if (find_group(op.rot->t_bounds, t) < 0) return TRDQ_ERR_TIMESTEP;
     if (op.M < 0 || op.ldx < op.rot->K || op.ldy < op.w->N) return TRDQ_ERR_SHAPE;
     if (op.M > 0 && (!op.X_bf16 || !op.codes || !op.scales || !op.Y_bf16)) return TRDQ_ERR_NULL;
@@ -608,7 +612,9 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
   }
   for (int i = 0; i < count; ++i) {
     const trdq_layer_op& op = ops[i];
-    trdq_status st = trdq_rotate_quantize(op.rot, t, op.X_bf16, op.ldx, op.M, op.codes, op.scales, stream);
+    trdq_status st = op.rot->dense ? trdq_rotate_dense_quantize(op.rot, t, op.X_bf16, op.ldx, op.M, op.codes, op.scales, op.workspace,
+                                                                op.workspace_bytes, stream)
+                                   : trdq_rotate_quantize(op.rot, t, op.X_bf16, op.ldx, op.M, op.codes, op.scales, stream);
     if (st != TRDQ_OK) return st;
     st = trdq_linear_act(op.w, t, op.codes, op.scales, op.M, op.bias_bf16, op.Y_bf16, op.ldy, op.act, stream);
     if (st != TRDQ_OK) return st;

@@ -48,7 +48,7 @@ class RotationSpec(C.Structure):
 class LayerOp(C.Structure):
     _fields_ = [("rot", C.c_void_p), ("w", C.c_void_p), ("X_bf16", C.c_void_p), ("ldx", C.c_int64), ("M", C.c_int32),
                 ("codes", C.c_void_p), ("scales", C.c_void_p), ("bias_bf16", C.c_void_p), ("Y_bf16", C.c_void_p),
-                ("ldy", C.c_int64), ("act", C.c_int32)]
+                ("ldy", C.c_int64), ("act", C.c_int32), ("workspace", C.c_void_p), ("workspace_bytes", C.c_uint64)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -432,15 +432,18 @@ class LayerList:
 
     def __init__(self):
         self._keep = []
+        self._extra = []
         self._ops = []
         self._array = None
 
-    def add(self, rot: Rotation, w: Weights, X_bf16, codes, scales, bias_bf16, Y_bf16, act: int = 0) -> None:
+    def add(self, rot: Rotation, w: Weights, X_bf16, codes, scales, bias_bf16, Y_bf16, act: int = 0, workspace=None) -> None:
         M = int(X_bf16.shape[0])
         assert X_bf16.stride(1) == 1 and Y_bf16.stride(1) == 1 and codes.is_contiguous()
         self._ops.append(LayerOp(rot._h, w._h, _ptr(X_bf16), int(X_bf16.stride(0)) if M > 1 else rot.K, M, _ptr(codes),
-                                 _ptr(scales), _ptr(bias_bf16), _ptr(Y_bf16), int(Y_bf16.stride(0)) if M > 1 else w.N, int(act)))
+                                 _ptr(scales), _ptr(bias_bf16), _ptr(Y_bf16), int(Y_bf16.stride(0)) if M > 1 else w.N, int(act),
+                                 _ptr(workspace), 0 if workspace is None else int(workspace.numel() * workspace.element_size())))
         self._keep.append((rot, w, X_bf16, codes, scales, bias_bf16, Y_bf16))
+        self._extra.append(workspace)
         self._array = None
 
     def __len__(self) -> int:

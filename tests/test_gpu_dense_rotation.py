@@ -216,3 +216,53 @@ def test_dense_rotation_full_size_sampled_rows():
     bad = check_dense_codes(codes[idx].cpu().numpy(), scales[idx].cpu().numpy(), x_rows, stored)
     assert trdq.trdq_device_status() == 0
     print(f"full size: {bad} of {rows.size * K} sampled codes off by one")
+
+
+def test_dense_rotation_through_the_layer_list():
+    """trdq_run_layers with a dense-block rotation: the op carries the workspace; results equal the stand-alone calls bit for bit,
+    a Hadamard op in the same list is unaffected, and a missing or short workspace is rejected before anything is launched."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(91)
+    K, N, M = 384, 256, 300
+    blocks = orthogonal_blocks(2, K // 128, 92)
+    bounds = WL.group_bounds(2)
+    drot = trdq.DenseRotation(K, bounds, blocks, None)
+    hrot = trdq.Rotation(K, bounds, (rng.integers(0, 2, (2, K)) * 2 - 1).astype(np.int8))
+    w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.03)
+    bias = to_dev_bf16(WL.to_bf16_bits(rng.standard_normal(N) * 0.1))
+    x = to_dev_bf16(acts(M, K, 93))
+    layers = trdq.LayerList()
+    outs = []
+    for rot in (drot, hrot, drot):
+        wts = trdq.trdq_prepare_weights(rot, to_dev_bf16(w_bits), 8)
+        codes = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        scales = torch.empty((M,), dtype=torch.float32, device="cuda")
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(trdq.trdq_rotate_dense_workspace(rot, M), dtype=torch.uint8, device="cuda") if rot is drot else None
+        layers.add(rot, wts, x, codes, scales, bias, y, act=1 if rot is hrot else 0, workspace=ws)
+        outs.append((rot, wts, codes, scales, y))
+    t = 600
+    trdq.trdq_run_layers(layers, t)
+    for rot, wts, codes, scales, y in outs:
+        if rot is drot:
+            c2, s2 = trdq.trdq_rotate_dense_quantize(rot, t, x)
+            y2 = trdq.trdq_linear(wts, t, c2, s2, bias)
+        else:
+            c2, s2 = trdq.trdq_rotate_quantize(rot, t, x)
+            y2 = trdq.trdq_linear_act(wts, t, c2, s2, bias, act=1)
+        assert torch.equal(c2, codes) and torch.equal(s2, scales) and torch.equal(y2, y)
+    stored = O.dense_stored_blocks(blocks[1], None)
+    check_dense_codes(outs[0][2].cpu().numpy(), outs[0][3].cpu().numpy(), WL.to_bf16_bits(bf16_to_f32_np(x).astype(np.float64)), stored)
+    bad = trdq.LayerList()
+    rot, wts, codes, scales, y = outs[0]
+    bad.add(rot, wts, x, codes, scales, bias, y)                       # no workspace
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_run_layers(bad, t)
+    assert e.value.status == 1
+    short = trdq.LayerList()
+    short.add(rot, wts, x, codes, scales, bias, y, workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_run_layers(short, t)
+    assert e.value.status == 8
+    assert trdq.trdq_device_status() == 0
