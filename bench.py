@@ -342,13 +342,42 @@ def run_ours(args, wl: WL.Workload):
     ts = wl.timesteps()
     n_ops = len(layers)
 
-    def step(i):
+    def step_direct(i):
         trdq.trdq_run_layers(layers, int(ts[i % len(ts)]))
 
     for i in range(max(args.warmup, 3)):
-        step(i)
+        step_direct(i)
     torch.cuda.synchronize()
     assert trdq.trdq_device_status() == 0
+
+    # One CUDA graph per time-step group (the kernels of a step depend on t only through its group: a group switch is a
+    # switch of graph); the step of the sampling loop replays the graph of its group.
+    graphs = {}
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        for t in ts:
+            g = trdq.trdq_find_group(wl.t_bounds, int(t))
+            if g in graphs:
+                continue
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                trdq.trdq_run_layers(layers, int(t))
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graphs[g] = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graphs[g]):
+                trdq.trdq_run_layers(layers, int(t))
+        groups_of_steps = [trdq.trdq_find_group(wl.t_bounds, int(t)) for t in ts]
+
+    def step(i):
+        if graphs:
+            graphs[groups_of_steps[i % len(ts)]].replay()
+        else:
+            step_direct(i)
+
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -442,7 +471,8 @@ def run_ours(args, wl: WL.Workload):
         "dtype": "int8" if wl.wbits == 8 else "int8xint4", "data": "synthetic",
         "config": {"workload": wl.name, "M": wl.M, "blocks": wl.blocks, "linears_per_step": n_ops, "groups": wl.num_groups,
                    "sampling_steps": wl.steps, "wbits": wl.wbits, "parallelism": f"replicas x{world} (rows independent)",
-                   "rotation": args.rotation,
+                   "rotation": args.rotation, "launch": "host" if args.no_graph else "one CUDA graph per time-step group",
+
                    "l2": "inputs larger than L2: every linear has its own X, codes, Y and weights"},
         "us_per_dit_step": ms_per_step * 1e3,
         "rotate_quantize_gbs": rq_gbs,
@@ -480,6 +510,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into the workload list (1 = DiT-XL/2 256px, M = 4096)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host instead of replaying one CUDA graph per time-step group")
     ap.add_argument("--rotation", default="hadamard", choices=["hadamard", "dense"],
                     help="hadamard: the headline path; dense: dense 128 x 128 blocks on the tensor cores (Eq. 6-8), no CPU baseline")
     args = ap.parse_args()
