@@ -189,6 +189,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
     }
   }
   griddep_launch_dependents();
+  // The weights are constants of the prepared object, so the weight halves of the first tile's first stages are requested
+  // before waiting for the kernel before (which produced the activation codes): their latency overlaps its tail.
+  const int prefetched = cluster_id < total_tiles ? min(C::kStages, num_kb) : 0;
+  if (threadIdx.x == 0) {
+    const uint32_t leader_full0 = map_to_cta(bar_full, 0);
+    const TileCoord tc0 = pair_tile_coord(p, cluster_id < total_tiles ? cluster_id : 0, BN);
+    for (int kb = 0; kb < prefetched; ++kb) {
+      const uint32_t full_s = leader_full0 + 8 * kb;
+      mbar_remote_arrive_expect_tx(full_s, C::kStageBytes);  // this CTA's whole stage; the activation half follows below
+      tma_load_2d_pair(smem_base + kb * C::kStageBytes + C::kABytes, &p.tmap_b, kb * kTileKBytes, tc0.n0 + rank * (BN / 2), full_s);
+    }
+  }
   griddep_wait();
 
   if (warp == 0) {
@@ -205,9 +217,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
           const uint32_t a_dst = smem_base + stage * C::kStageBytes;
           const uint32_t b_dst = a_dst + C::kABytes;
           const uint32_t full_s = leader_full + 8 * stage;
-          mbar_remote_arrive_expect_tx(full_s, C::kStageBytes);
+          const bool b_in_flight = tile == cluster_id && kb < prefetched;
+          if (!b_in_flight) mbar_remote_arrive_expect_tx(full_s, C::kStageBytes);
           tma_load_2d_pair(a_dst, &p.tmap_a[tc.seg], kb * kTileKBytes, tc.m0 + rank * kTileM, full_s);
-          tma_load_2d_pair(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0 + rank * (BN / 2), full_s);
+          if (!b_in_flight) tma_load_2d_pair(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0 + rank * (BN / 2), full_s);
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1;
