@@ -140,3 +140,44 @@ def test_greedy_rotation_block_matches_oracle(lib):
     with pytest.raises(trdq.TrdqError) as e:
         trdq.trdq_greedy_rotation_block(bad, gauss)
     assert e.value.status == 5
+
+
+def test_dense_rotation_and_fusion_calls_validate_on_the_host(lib):
+    """The newer entry points reject bad arguments before any CUDA call: the dense-block specification (shape, bounds,
+    smoothing values, singular or non-finite blocks), and null handles of the dense, norm-fused and activation calls."""
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(3)
+    q, _ = np.linalg.qr(rng.standard_normal((128, 128)))
+    blocks = np.stack([q, q.T]).astype(np.float32)[None]           # K = 256, one group
+
+    def status_of(K=256, bounds=(0, 1000), blk=blocks, smooth=None):
+        try:
+            trdq.DenseRotation(K, list(bounds), blk, smooth)
+        except trdq.TrdqError as e:
+            return e.status
+        return 0
+
+    b = np.ascontiguousarray([0, 1000], np.int32)
+    f = blocks.ctypes.data_as(C.POINTER(C.c_float))
+    h = C.c_void_p()
+    assert lib.trdq_rotation_create_dense(200, 1, b.ctypes.data_as(C.POINTER(C.c_int32)), f, None, C.byref(h)) == 2
+    assert lib.trdq_rotation_create_dense(256, 0, b.ctypes.data_as(C.POINTER(C.c_int32)), f, None, C.byref(h)) == 5
+    assert lib.trdq_rotation_create_dense(256, 1, None, f, None, C.byref(h)) == 1
+    assert status_of(bounds=(10, 10)) == 5
+    assert status_of(smooth=np.full((1, 256), -1.0, np.float32)) == 5
+    singular = blocks.copy()
+    singular[0, 1, :, 3] = singular[0, 1, :, 40]
+    assert status_of(blk=singular) == 5
+    inf = blocks.copy()
+    inf[0, 0, 7, 7] = np.inf
+    assert status_of(blk=inf) == 5
+    import torch
+    if not torch.cuda.is_available():
+        assert status_of() in (7, 8)                                 # a valid specification needs a device and says so
+    n = C.c_uint64()
+    assert lib.trdq_rotate_dense_workspace(None, 16, C.byref(n)) == 1
+    assert lib.trdq_rotate_dense_quantize(None, 0, None, 0, 0, None, None, None, 0, None) == 1
+    assert lib.trdq_norm_rotate_quantize(None, 0, None, 0, 0, None, None, 1, C.c_float(1e-6), None, None, None) == 1
+    assert lib.trdq_linear_act(None, 0, None, None, 0, None, None, 0, 7, None) == 2      # unknown activation
+    assert lib.trdq_linear_act(None, 0, None, None, 0, None, None, 0, 1, None) == 1
+    assert lib.trdq_run_layers(None, 3, 0, None) == 1 and lib.trdq_run_layers(None, 0, 0, None) == 0
