@@ -221,7 +221,7 @@ def kernel_pass_ms(layers, wl, which: str, reps: int):
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
+    with torch.cuda.graph(graph, capture_error_mode="thread_local"):
         issue()
     for _ in range(3):
         graph.replay()
@@ -365,7 +365,7 @@ def run_ours(args, wl: WL.Workload):
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
             graphs[g] = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graphs[g]):
+            with torch.cuda.graph(graphs[g], capture_error_mode="thread_local"):
                 trdq.trdq_run_layers(layers, int(t))
         groups_of_steps = [trdq.trdq_find_group(wl.t_bounds, int(t)) for t in ts]
 

@@ -102,7 +102,7 @@ def main():
         # one pass over all buffer sets captured in a CUDA graph: launches are back to back on the
         # device, so small shapes are not limited by the host's launch rate
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
             for i in range(args.sets):
                 run(i)
         graph.replay()
