@@ -421,7 +421,10 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
     tiles_m += p.pair_tiles_m[s];
   }
   if (tiles_m == 0) return TRDQ_OK;
-  // tile width by the same wave model as the single-CTA kernel, over the resident clusters
+  // Tile width: waves of resident clusters times the time of one tile.  The kernel is bound by operand delivery from L2,
+  // so a tile costs what it loads, (256 + BN) panel rows of K bytes; wider tiles load less per multiply-add.  Checked
+  // against a sweep of all three widths over the layer shapes at M = 4096 ... 32768: the model picks the fastest width or
+  // one within 2 % of it (the earlier model, waves x (BN + 24), left 4 - 15 % on the table at M >= 16384).
   int best = -1;
   double best_cost = 1e300;
   int clusters_of[kNumTileN];
@@ -431,7 +434,7 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
     if (clusters_of[i] <= 0) continue;
     const int64_t tiles = tiles_m * ((w->N + bn - 1) / bn);
     const int64_t waves = (tiles + clusters_of[i] - 1) / clusters_of[i];
-    const double cost = static_cast<double>(waves) * (bn + 24.0);
+    const double cost = static_cast<double>(waves) * (256.0 + bn);
     if (cost < best_cost) {
       best_cost = cost;
       best = i;
