@@ -23,8 +23,10 @@
  *     memory.  bf16 tensors are passed as `const void*` / `void*` to 2-byte elements.
  *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = the legacy default stream).
  *   - All device work is enqueued asynchronously on `stream`; no entry point
- *     synchronises unless its comment says so.  The online calls (trdq_rotate_quantize,
- *     trdq_linear, trdq_linear_cfg, trdq_gemm_i32) allocate no memory.
+ *     synchronises unless its comment says so.  The online calls (trdq_rotate_quantize and
+ *     its _asym, _dense and norm-fused forms, trdq_linear and its _cfg, _act, _asym and split-K
+ *     forms, trdq_run_layers, trdq_gemm_i32) allocate no memory; trdq_prepare_weights with a
+ *     dense-block rotation is the one call that waits for its own work (it frees a scratch buffer).
  *   - The caller owns every tensor it passes.  The library owns only the opaque
  *     trdq_rotation / trdq_weights objects until their _destroy call.
  *   - Errors are reported by return code only; the library never aborts, traps or
@@ -56,7 +58,7 @@ typedef enum trdq_status {
   TRDQ_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (no device, launch error, ...) */
   TRDQ_ERR_NOMEM = 8,     /* host or device allocation failed */
   TRDQ_ERR_TIMEOUT = 9,   /* a bounded device-side wait expired (see trdq_device_status) */
-  TRDQ_ERR_MISMATCH = 10, /* objects passed together were built for different K / groups */
+  TRDQ_ERR_MISMATCH = 10, /* objects passed together were built for different K / groups, or the rotation's kind does not fit the call */
   TRDQ_ERR_SCRATCH = 11   /* the problem needs more than the library's built-in scratch area (trdq_linear_splitk_static) */
 } trdq_status;
 
