@@ -144,7 +144,21 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
     prefetch_tensormap(&p.tmap_out[1]);
   }
   griddep_launch_dependents();
-  griddep_wait();  // codes, scales and weights may come from the kernel before; Y may still be read by it
+  // The weights are constants of the prepared object: the weight tiles of the first tile's first stages are requested
+  // before waiting for the kernel before (which produced the activation codes), so their latency overlaps its tail.
+  int prefetched = 0;
+  if (static_cast<int>(blockIdx.x) < total_tiles) {
+    const TileCoord tc0 = tile_coord(p, blockIdx.x, BN);
+    const int kb0 = tc0.split * p.kb_per_split;
+    prefetched = min(C::kStages, min(kb0 + p.kb_per_split, num_kb_all) - kb0);
+    if (threadIdx.x == 0) {
+      for (int i = 0; i < prefetched; ++i) {
+        mbar_arrive_expect_tx(bar_full + 8 * i, C::kStageBytes);  // the whole stage; the activation tile follows below
+        tma_load_2d(smem_base + i * C::kStageBytes + C::kABytes, &p.tmap_b, (kb0 + i) * kTileKBytes, tc0.n0, bar_full + 8 * i);
+      }
+    }
+  }
+  griddep_wait();  // codes and scales may come from the kernel before; Y may still be read by it
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -160,9 +174,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
           w.wait(bar_empty + 8 * stage, phase ^ 1);
           const uint32_t a_dst = smem_base + stage * C::kStageBytes;
           const uint32_t b_dst = a_dst + C::kABytes;
-          mbar_arrive_expect_tx(bar_full + 8 * stage, C::kStageBytes);
+          const bool b_in_flight = tile == static_cast<int>(blockIdx.x) && kb - kb0 < prefetched;
+          if (!b_in_flight) mbar_arrive_expect_tx(bar_full + 8 * stage, C::kStageBytes);
           tma_load_2d(a_dst, &p.tmap_a[tc.seg], kb * kTileKBytes, tc.m0, bar_full + 8 * stage);
-          tma_load_2d(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0, bar_full + 8 * stage);
+          if (!b_in_flight) tma_load_2d(b_dst, &p.tmap_b, kb * kTileKBytes, tc.n0, bar_full + 8 * stage);
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1;
