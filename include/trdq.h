@@ -136,7 +136,7 @@ trdq_status trdq_weights_view(const trdq_weights* w, int32_t g, const void** Wq,
 trdq_status trdq_weights_export(const trdq_weights* w, int32_t g, void* codes_out, float* scales_out, void* stream);
 
 /* Online activation path G_t(X) followed by dynamic per-token quantization (Sec. 3.1 Eq. 1-2,
- * Sec. 3.2 "calculating quantization parameters online"):
+ * Sec. 3.2: the activation scales are computed online, per token):
  *   v[m, :]   = (x[m, :] o act_g) . BlockDiag(H_128), fp32 butterflies in the order h = 1, 2, ..., 64
  *   scales[m] = absmax_k |v[m, k]| / 127
  *   codes[m,k]= rne(v[m, k] * fl32(127 / absmax))     (all-zero row: scale 0, codes 0)
@@ -191,6 +191,10 @@ trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* c
  *     call is trdq_linear.
  *   - The first call on a device looks up the array's device address (once per device, with that device
  *     current) and configures the kernels; make that first call during start-up, before any stream capture.
+ *   - "Allocates nothing" holds once the library's GEMM code is resident on the device: the array is part of
+ *     that code image and the driver reserves its 8 MiB when the image is first used there (any trdq_linear*
+ *     call, or trdq_prepare_weights with 8-bit weights, does that).  A server that hands the rest of the
+ *     device to its own pool must make one such call first, or the load itself fails with TRDQ_ERR_CUDA.
  *   - All calls share the one array, and it keeps the last call's contents.  That is harmless for
  *     calls that run one after another (every value read is written by the same call first), but two
  *     calls that overlap on the GPU -- different streams, or concurrent host threads -- race on it:

@@ -9,15 +9,15 @@
 //   * Sec. 3.1, Eq. 1-2: uniform integer quantizer with nearest rounding, used in
 //     its symmetric signed 8-bit form (zero-point 0, scale = absmax / 127);
 //     per-token scales for activations and per-output-channel scales for weights
-//     ("per-token quantization for activations and per-channel ... for weights").
+//     (the granularity paragraph of Sec. 3.1).
 //   * Sec. 3.1, Eq. 4: channel scaling vector Delta.  Following Eq. 10 the online
 //     side MULTIPLIES X by Delta_t and the offline side multiplies W by 1/Delta_t.
 //   * Sec. 3.2, Eq. 8: block-diagonal orthogonal rotation, blocks of 2^n x 2^n;
 //     here n = 7 and every block is diag(d) * H_128 / sqrt(128) with H_128 the
 //     Sylvester-Walsh-Hadamard matrix and d a +-1 vector per time-step group.
 //   * Sec. 3.2, Eq. 10: F_t(X, W) = G_t(X) . H_t(W) with the parameter set chosen
-//     by the current time-step; "dynamic quantization ... calculating quantization
-//     parameters online" for the activations.
+//     by the current time-step; the activation scales are computed online from each
+//     token's own rotated values (Sec. 3.2, paragraph after Eq. 9).
 //
 // Parity notes.  The quantizer, the integer GEMM and the dequantising epilogue are
 // pinned by the tests against closed forms and brute force.  Two things are

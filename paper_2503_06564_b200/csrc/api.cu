@@ -15,15 +15,17 @@ namespace trdq {
 __device__ uint32_t g_status_word;
 
 uint32_t* device_status_word() {
-  static uint32_t* cached[64] = {};
+  static PerDevice<uint32_t*> cached;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!cached[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  uint32_t* addr = cached.get(dev);
+  if (!addr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-    cached[dev] = static_cast<uint32_t*>(p);
+    addr = static_cast<uint32_t*>(p);
+    cached.set(dev, addr);
   }
-  return cached[dev];
+  return addr;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -90,6 +92,27 @@ trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool aligned_to(const void* p, uintptr_t bytes) { return (reinterpret_cast<uintptr_t>(p) & (bytes - 1)) == 0; }
+
+// Objects hold device memory and tensor maps of the device they were created on; a call made with another device
+// current would launch there with pointers of the first one.
+static bool on_current_device(int device) {
+  int cur = -1;
+  return cudaGetDevice(&cur) == cudaSuccess && cur == device;
+}
+
+// Pointer, stride and alignment rules of ONE row segment of a linear call.  Every linear entry point goes through
+// this function, so a bad argument is reported on the host and never reaches a kernel (which would read sx[m] as
+// a float, bias[n] as bf16 and store 16-byte pieces of Y).  `raw`: int32 accumulators out, no scales.
+static trdq_status check_linear_segment(const trdq_weights* w, const void* codes, const float* scales, const void* out, int64_t ld,
+                                        bool raw) {
+  if (!codes || !out || (!raw && !scales)) return TRDQ_ERR_NULL;
+  if (ld < w->N) return TRDQ_ERR_SHAPE;
+  if (ld % (raw ? 4 : 8) != 0 || !aligned16(codes) || !aligned16(out) || (!raw && !aligned_to(scales, 4))) return TRDQ_ERR_ALIGN;
+  return TRDQ_OK;
+}
+
+static trdq_status check_bias(const void* bias_bf16) { return bias_bf16 && !aligned_to(bias_bf16, 2) ? TRDQ_ERR_ALIGN : TRDQ_OK; }
 
 static int find_group(const std::vector<int32_t>& bounds, int32_t t) {
   const int G = static_cast<int>(bounds.size()) - 1;
@@ -275,6 +298,7 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
   if (wbits != 8 && wbits != 4) return TRDQ_ERR_WBITS;
   if (N <= 0 || N % 16 != 0) return TRDQ_ERR_SHAPE;
   if (!aligned16(W_bf16)) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const int K = rot->K, G = rot->num_groups;
 
   trdq_weights* w = new (std::nothrow) trdq_weights;
@@ -427,6 +451,7 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
   if (!X_bf16 || !codes || !scales) return TRDQ_ERR_NULL;
   if (ldx < rot->K) return TRDQ_ERR_SHAPE;
   if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const float* vec = rot->act_vec + static_cast<size_t>(g) * rot->K;
   if (rot->perm) {
     const cudaError_t e2 = launch_rotate2_quantize(X_bf16, ldx, M, rot->K, vec, rot->perm + static_cast<size_t>(g) * rot->K,
@@ -454,6 +479,7 @@ trdq_status trdq_norm_rotate_quantize(const trdq_rotation* rot, int32_t t, const
   if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u) ||
       (shift_bf16 && !aligned16(shift_bf16)) || (scale_bf16 && !aligned16(scale_bf16)))
     return TRDQ_ERR_ALIGN;
+  if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const cudaError_t e = launch_norm_rotate_quantize(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, shift_bf16,
                                                     scale_bf16, rows_per_sample, eps, codes, scales, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
@@ -468,16 +494,15 @@ static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t*
   if (g < 0) return TRDQ_ERR_TIMESTEP;
   if (raw && w->wbits != 8) return TRDQ_ERR_WBITS;
   GemmSegment seg[2];
-  const int ld_mult = raw ? 4 : 8;
   for (int s = 0; s < 2; ++s) {
     seg[s] = GemmSegment{codes[s], raw ? nullptr : scales[s], Y[s], ld[s], M[s]};
     if (M[s] == 0) continue;
-    if (!codes[s] || !Y[s] || (!raw && !scales[s])) return TRDQ_ERR_NULL;
-    if (ld[s] < w->N) return TRDQ_ERR_SHAPE;
-    if (ld[s] % ld_mult != 0 || !aligned16(codes[s]) || !aligned16(Y[s])) return TRDQ_ERR_ALIGN;
+    const trdq_status st = check_linear_segment(w, codes[s], raw ? nullptr : scales[s], Y[s], ld[s], raw);
+    if (st != TRDQ_OK) return st;
   }
   if (M[0] == 0 && M[1] == 0) return TRDQ_OK;
-  if (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)) return TRDQ_ERR_ALIGN;
+  if (check_bias(bias) != TRDQ_OK) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   if (w->wbits == 8) return launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream), act);
   return launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream), act);
 }
@@ -526,9 +551,11 @@ trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* c
   if (splits <= 1) return trdq_linear(w, t, codes, scales, M, bias_bf16, Y_bf16, ldy, stream);
   const int g = find_group(w->t_bounds, t);
   if (g < 0) return TRDQ_ERR_TIMESTEP;
-  if (!codes || !scales || !Y_bf16 || !workspace) return TRDQ_ERR_NULL;
-  if (ldy < w->N) return TRDQ_ERR_SHAPE;
-  if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16) || !aligned16(workspace)) return TRDQ_ERR_ALIGN;
+  if (!workspace) return TRDQ_ERR_NULL;
+  const trdq_status chk = check_linear_segment(w, codes, scales, Y_bf16, ldy, false);
+  if (chk != TRDQ_OK) return chk;
+  if (!aligned16(workspace) || check_bias(bias_bf16) != TRDQ_OK) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   if (workspace_bytes < static_cast<uint64_t>(splits) * static_cast<uint64_t>(M) * static_cast<uint64_t>(w->N) * 4u) return TRDQ_ERR_NOMEM;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
   return launch_gemm_w8_splitk(w, g, seg, bias_bf16, splits, static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream));
@@ -542,9 +569,10 @@ trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const in
   if (splits <= 1) return trdq_linear(w, t, codes, scales, M, bias_bf16, Y_bf16, ldy, stream);
   const int g = find_group(w->t_bounds, t);
   if (g < 0) return TRDQ_ERR_TIMESTEP;
-  if (!codes || !scales || !Y_bf16) return TRDQ_ERR_NULL;
-  if (ldy < w->N) return TRDQ_ERR_SHAPE;
-  if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16)) return TRDQ_ERR_ALIGN;
+  const trdq_status chk = check_linear_segment(w, codes, scales, Y_bf16, ldy, false);
+  if (chk != TRDQ_OK) return chk;
+  if (check_bias(bias_bf16) != TRDQ_OK) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
   return launch_gemm_w8_splitk_static(w, g, seg, bias_bf16, splits, static_cast<cudaStream_t>(stream));
 }
@@ -562,6 +590,7 @@ trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const
   if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u) ||
       (reinterpret_cast<uintptr_t>(zero_points) & 3u))
     return TRDQ_ERR_ALIGN;
+  if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const cudaError_t e = launch_rotate_quantize_asym(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, codes, scales,
                                                     zero_points, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
@@ -575,9 +604,11 @@ trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* co
   const int g = find_group(w->t_bounds, t);
   if (g < 0) return TRDQ_ERR_TIMESTEP;
   if (M == 0) return TRDQ_OK;
-  if (!codes || !scales || !zero_points || !Y_bf16) return TRDQ_ERR_NULL;
-  if (ldy < w->N) return TRDQ_ERR_SHAPE;
-  if (ldy % 8 != 0 || !aligned16(codes) || !aligned16(Y_bf16)) return TRDQ_ERR_ALIGN;
+  if (!zero_points) return TRDQ_ERR_NULL;
+  const trdq_status chk = check_linear_segment(w, codes, scales, Y_bf16, ldy, false);
+  if (chk != TRDQ_OK) return chk;
+  if (!aligned_to(zero_points, 4) || check_bias(bias_bf16) != TRDQ_OK) return TRDQ_ERR_ALIGN;
+  if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   GemmSegment seg[2] = {GemmSegment{reinterpret_cast<const int8_t*>(codes), scales, Y_bf16, ldy, M}, GemmSegment{nullptr, nullptr, nullptr, ldy, 0}};
   const int32_t* zp[2] = {zero_points, nullptr};
   return launch_gemm_w8_asym(w, g, seg, zp, bias_bf16, static_cast<cudaStream_t>(stream));
@@ -598,7 +629,7 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
   for (int i = 0; i < count; ++i) {
     const trdq_layer_op& op = ops[i];
     if (!op.rot || !op.w) return TRDQ_ERR_NULL;
-    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds) return TRDQ_ERR_MISMATCH;
+    if (op.rot->K != op.w->K || op.rot->t_bounds != op.w->t_bounds || op.rot->device != op.w->device) return TRDQ_ERR_MISMATCH;
     if (op.rot->dense && op.M > 0) {
       if (!op.workspace) return TRDQ_ERR_NULL;
       if (op.workspace_bytes < rotate_dense_workspace_bytes(op.M, op.rot->K)) return TRDQ_ERR_NOMEM;
@@ -606,7 +637,8 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
     if (find_group(op.rot->t_bounds, t) < 0) return TRDQ_ERR_TIMESTEP;
     if (op.M < 0 || op.ldx < op.rot->K || op.ldy < op.w->N) return TRDQ_ERR_SHAPE;
     if (op.M > 0 && (!op.X_bf16 || !op.codes || !op.scales || !op.Y_bf16)) return TRDQ_ERR_NULL;
-    if (op.ldx % 8 != 0 || op.ldy % 8 != 0 || !aligned16(op.X_bf16) || !aligned16(op.codes) || !aligned16(op.Y_bf16))
+    if (op.ldx % 8 != 0 || op.ldy % 8 != 0 || !aligned16(op.X_bf16) || !aligned16(op.codes) || !aligned16(op.Y_bf16) ||
+        !aligned_to(op.scales, 4) || check_bias(op.bias_bf16) != TRDQ_OK)
       return TRDQ_ERR_ALIGN;
     if (op.act != TRDQ_ACT_NONE && op.act != TRDQ_ACT_GELU_TANH) return TRDQ_ERR_SHAPE;
   }

@@ -318,13 +318,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
 template <int BN, int MODE>
 cudaError_t launch_one(const GemmParams& p, int grid, cudaStream_t stream) {
   using C = Cfg<BN>;
-  static bool configured[16] = {};
+  static PerDeviceFlag configured;
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  if (!configured.get(dev)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_w8a8_kernel<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured[dev] = true;
+    configured.set(dev, true);
   }
   return launch_overlapped(gemm_w8a8_kernel<BN, MODE>, dim3(grid), dim3(kThreads), C::kSmemBytes, stream, p);
 }
@@ -576,18 +576,18 @@ static __device__ __align__(256) int32_t g_static_splitk_scratch[TRDQ_STATIC_SCR
 // for the runtime, not an address a kernel could use, so the address is asked for once per device
 // (with that device current) and remembered.
 static int32_t* static_scratch_address() {
-  static int32_t* cached[64] = {};
+  static PerDevice<int32_t*> cached;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!cached[dev]) {
-    int32_t* ptr = nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  int32_t* ptr = cached.get(dev);
+  if (!ptr) {
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_splitk_scratch) != cudaSuccess || !ptr) {
       cudaGetLastError();
       return nullptr;
     }
-    cached[dev] = ptr;
+    cached.set(dev, ptr);
   }
-  return cached[dev];
+  return ptr;
 }
 
 trdq_status launch_gemm_w8_splitk_static(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,

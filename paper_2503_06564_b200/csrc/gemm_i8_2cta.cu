@@ -380,14 +380,15 @@ cudaError_t launch_pair(const Gemm2Params& p, int clusters, cudaStream_t stream)
 // Clusters of two CTAs that can be resident at once (at most SMs / 2; fewer if a GPC has an odd SM count).
 template <int BN>
 int max_clusters(int dev) {
-  static int cached[16] = {};
-  if (dev < 0 || dev >= 16) return 0;
-  if (cached[dev] == 0) {
+  static PerDevice<int> cached;
+  if (dev < 0 || dev >= kMaxDevices) return 0;
+  int known = cached.get(dev);
+  if (known == 0) {
     using C = Cfg2<BN>;
     if (cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_w8a8_pair_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess) {
       cudaGetLastError();
-      cached[dev] = -1;
+      cached.set(dev, -1);
       return 0;
     }
     cudaLaunchConfig_t cfg = {};
@@ -397,12 +398,13 @@ int max_clusters(int dev) {
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, gemm_w8a8_pair_kernel<BN, false>, &cfg) != cudaSuccess || n <= 0) {
       cudaGetLastError();
-      cached[dev] = -1;
+      cached.set(dev, -1);
       return 0;
     }
-    cached[dev] = n;
+    known = n;
+    cached.set(dev, n);
   }
-  return cached[dev] > 0 ? cached[dev] : 0;
+  return known > 0 ? known : 0;
 }
 
 }  // namespace

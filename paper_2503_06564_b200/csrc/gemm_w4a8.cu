@@ -413,13 +413,13 @@ trdq_status launch_gemm_w4(const trdq_weights* w, int g, const GemmSegment seg[2
   const int smem_bytes = kFixedSmemBytes + (p.mult_in_smem ? groups * kTileNW4 * 4 : 0);
   const int64_t total = tiles_m * p.tiles_n;
   const int grid = static_cast<int>(total < sms ? total : sms);
-  static bool configured[16] = {};
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  static PerDeviceFlag configured;
+  if (!configured.get(dev)) {
     const int max_smem = kFixedSmemBytes + kMaxSmemGroups * kTileNW4 * 4;
     if (cudaFuncSetAttribute(gemm_w4a8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_w4a8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
       return TRDQ_ERR_CUDA;
-    configured[dev] = true;
+    configured.set(dev, true);
   }
   const cudaError_t e = act ? launch_overlapped(gemm_w4a8_kernel<true>, dim3(grid), dim3(kThreads), smem_bytes, stream, p)
                             : launch_overlapped(gemm_w4a8_kernel<false>, dim3(grid), dim3(kThreads), smem_bytes, stream, p);

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <vector>
 
 #include "../../include/trdq.h"
@@ -52,6 +53,20 @@ struct trdq_weights {
 };
 
 namespace trdq {
+
+// Per-device memo for set-up done by the first call on a device (kernel attributes, symbol addresses, occupancy
+// queries).  Several host threads may make that first call at once: repeating the set-up is harmless, a torn
+// read of the memo is not, hence the atomics.  A zero value means "not done yet".
+constexpr int kMaxDevices = 64;
+template <typename T>
+struct PerDevice {
+  std::atomic<T> slot[kMaxDevices];
+  T get(int dev) const { return dev >= 0 && dev < kMaxDevices ? slot[dev].load(std::memory_order_acquire) : T(); }
+  void set(int dev, T v) {
+    if (dev >= 0 && dev < kMaxDevices) slot[dev].store(v, std::memory_order_release);
+  }
+};
+using PerDeviceFlag = PerDevice<bool>;
 
 uint32_t* device_status_word();  // device address of the status word of the current device (nullptr on failure)
 

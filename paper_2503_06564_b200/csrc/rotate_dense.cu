@@ -462,13 +462,13 @@ __global__ void __launch_bounds__(256) quantize_rows_w4_kernel(const float* __re
 }
 
 template <typename Kernel>
-cudaError_t launch_pass(Kernel kernel, int smem_bytes, bool* configured, const DenseParams& p, dim3 grid, cudaStream_t stream) {
+cudaError_t launch_pass(Kernel kernel, int smem_bytes, PerDeviceFlag& configured, const DenseParams& p, dim3 grid, cudaStream_t stream) {
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  if (!configured.get(dev)) {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    configured[dev] = true;
+    configured.set(dev, true);
   }
   return launch_overlapped(kernel, grid, dim3(kThreads), smem_bytes, stream, p);
 }
@@ -499,7 +499,7 @@ trdq_status launch_rotate_dense_quantize(const trdq_rotation* rot, int g, const 
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return TRDQ_ERR_CUDA;
-  static bool configured0[16] = {}, configured1[16] = {};
+  static PerDeviceFlag configured0, configured1;
   // Both passes cover all token tiles in one launch each.  (Cutting the rows into L2-sized chunks, each with its own
   // pair of launches, was measured: the second read then hits L2, but the extra launches cost what the hits save.)
   const int tiles = (M + kRows - 1) / kRows;

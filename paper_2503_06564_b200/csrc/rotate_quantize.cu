@@ -651,11 +651,11 @@ cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, 
     int dev2 = 0, sms2 = 148;
     cudaGetDevice(&dev2);
     cudaDeviceGetAttribute(&sms2, cudaDevAttrMultiProcessorCount, dev2);
-    static bool configured2[16] = {};
-    if (dev2 >= 0 && dev2 < 16 && !configured2[dev2]) {
+    static PerDeviceFlag configured2;
+    if (!configured2.get(dev2)) {
       const cudaError_t e = cudaFuncSetAttribute(rotate2_quantize_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
       if (e != cudaSuccess) return e;
-      configured2[dev2] = true;
+      configured2.set(dev2, true);
     }
     const int tiles2 = (M + rows2 - 1) / rows2;
     return launch_overlapped(rotate2_quantize_rows_kernel<2>, dim3(min(tiles2, sms2 * 2)), dim3(threads2), smem2, stream,
@@ -670,12 +670,12 @@ cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  static bool configured[16] = {};
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  static PerDeviceFlag configured;
+  if (!configured.get(dev)) {
     cudaError_t e = cudaFuncSetAttribute(rotate2_quantize_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(rotate2_quantize_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
     if (e != cudaSuccess) return e;
-    configured[dev] = true;
+    configured.set(dev, true);
   }
   const int num_tiles = (M + rows - 1) / rows;
   const int ctas_per_sm = max(1, min(2048 / threads, static_cast<int>((200 * 1024) / (smem + 1024))));

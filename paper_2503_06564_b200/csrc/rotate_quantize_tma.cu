@@ -261,14 +261,14 @@ trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t 
   if (!p.status) return TRDQ_ERR_CUDA;
   const size_t smem = 1024 + 2 * static_cast<size_t>(R) * K * 2 + static_cast<size_t>(R) * K + static_cast<size_t>(K) * 4 +
                       3 * static_cast<size_t>(R) * 4 + 64;
-  static bool configured[16] = {};
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  static PerDeviceFlag configured;
+  if (!configured.get(dev)) {
     if (cudaFuncSetAttribute(rotate_quantize_tma_kernel<kMaxComputeThreads, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              227 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(rotate_quantize_tma_kernel<kSmallComputeThreads, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              113 * 1024) != cudaSuccess)
       return TRDQ_ERR_CUDA;
-    configured[dev] = true;
+    configured.set(dev, true);
   }
   const bool small = false;  // two smaller CTAs per SM measured slower on 9- and 18-block rows, as did twelve compute warps with a one-stage ring
   if (smem > (small ? 113u : 227u) * 1024) return TRDQ_ERR_SHAPE;

@@ -52,19 +52,23 @@ def test_dit_xl2_256px_all_layers(layer_idx):
     _run_layer(WL.WORKLOADS[1], layer_idx, t=980)
 
 
-def test_dit_xl2_512px_fc2():
-    """M = 16384, K = 4608: the widest rows, through the one-thread-per-block rotate kernel and the CTA-pair GEMM."""
-    _run_layer(WL.WORKLOADS[2], 3, t=400, sample=256)
+@pytest.mark.parametrize("layer_idx", [0, 1, 2, 3])
+def test_dit_xl2_512px_all_layers(layer_idx):
+    """M = 16384, every layer shape (K = 1152 rows and the K = 4608 rows of fc2), one time-step per group across the layers."""
+    _run_layer(WL.WORKLOADS[2], layer_idx, t=(400, 0, 999, 600)[layer_idx], sample=256)
 
 
-def test_pixart_1024px_qkv_and_cross_attention():
+@pytest.mark.parametrize("layer_idx", [0, 1, 2, 3, 4, 5])
+def test_pixart_1024px_all_layers_and_cross_attention(layer_idx):
+    """M = 32768 on the four block linears; the cross-attention K and V projections on their 960 text rows (all rows)."""
     wl = WL.WORKLOADS[3]
-    _run_layer(wl, 0, t=10, sample=256)      # M = 32768, 1152 -> 3456
-    _run_layer(wl, 4, t=740, sample=960)     # cross-attention K projection: 960 text rows, 4096 -> 1152, all rows
+    _run_layer(wl, layer_idx, t=(10, 260, 510, 999, 740, 250)[layer_idx], sample=960 if layer_idx >= 4 else 256)
 
 
-def test_video_dit_w4a8_fc1():
-    _run_layer(WL.WORKLOADS[4], 2, t=700, sample=256)   # M = 16384, int4 weights, 1152 -> 4608
+@pytest.mark.parametrize("layer_idx", [0, 1, 2, 3])
+def test_video_dit_w4a8_all_layers(layer_idx):
+    """M = 16384, int4 weights; fc2 has 36 scale groups along K."""
+    _run_layer(WL.WORKLOADS[4], layer_idx, t=(700, 0, 350, 999)[layer_idx], sample=256)
 
 
 def test_run_layers_follows_the_time_step_schedule():

@@ -393,3 +393,65 @@ def test_maximum_k(wbits):
         y_ref = O.linear_w4_rows(q_ref, sx_ref, pk_ref, sw4_ref, None, rows)
     check_output(bf16_to_f32_np(y), y_ref)
     assert trdq.trdq_device_status() == 0
+
+
+def test_every_linear_entry_point_validates_on_the_host():
+    """Bad pointers, strides and time-steps are reported by the host code of every linear entry point (the plain one,
+    the two split-K forms and the asymmetric one) before anything is launched: the output stays untouched and the
+    device healthy.  Called through the C ABI directly so that misaligned addresses can be passed."""
+    import ctypes as C
+    import torch
+    from paper_2503_06564_b200 import trdq
+    lib = trdq.lib()
+    N, K, M = 1152, 8192, 128                        # a shape for which split-K is chosen, so those paths do their own checks
+    rot, wts, _, bias_bits, _ = _setup(N, K, 2, seed=21)
+    x_bits = _acts(M, K, 22)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, to_dev_bf16(x_bits))
+    bias = to_dev_bf16(bias_bits)
+    assert trdq.trdq_linear_splitk_workspace(wts, M)[0] > 1
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty((8 * M * N * 4,), dtype=torch.uint8, device="cuda")
+    zp = torch.zeros((M,), dtype=torch.int32, device="cuda")
+    h, st = wts._h, trdq._stream()
+    c, sc, b, yp, wp, z = (t.data_ptr() for t in (codes, scales, bias, y, ws, zp))
+
+    def calls(c=c, sc=sc, b=b, yp=yp, ldy=N, t=0, M=M):
+        return {
+            "linear": lib.trdq_linear(h, t, c, sc, M, b, yp, ldy, st),
+            "act": lib.trdq_linear_act(h, t, c, sc, M, b, yp, ldy, 0, st),
+            "splitk": lib.trdq_linear_splitk(h, t, c, sc, M, b, yp, ldy, wp, ws.numel(), st),
+            "static": lib.trdq_linear_splitk_static(h, t, c, sc, M, b, yp, ldy, st),
+            "asym": lib.trdq_linear_asym(h, t, c, sc, z, M, b, yp, ldy, st),
+        }
+
+    def all_equal(result, status):
+        assert set(result.values()) == {status}, result
+
+    all_equal(calls(M=-1), 2)                 # negative row count
+    all_equal(calls(t=1000), 4)               # time-step outside the covered range
+    all_equal(calls(t=-1), 4)
+    all_equal(calls(c=None), 1)
+    all_equal(calls(sc=None), 1)
+    all_equal(calls(yp=None), 1)
+    all_equal(calls(ldy=N - 8), 2)            # rows of Y would overlap
+    all_equal(calls(ldy=N + 4), 3)            # rows of Y not 16-byte aligned
+    all_equal(calls(c=c + 8), 3)
+    all_equal(calls(yp=yp + 2), 3)
+    all_equal(calls(sc=sc + 2), 3)            # the kernels read sx[m] as a 4-byte float
+    all_equal(calls(sc=sc + 1), 3)
+    all_equal(calls(b=b + 1), 3)              # ... and bias[n] as a 2-byte bf16
+    assert lib.trdq_linear_splitk(h, 0, c, sc, M, b, yp, N, wp + 4, ws.numel(), st) == 3
+    assert lib.trdq_linear_splitk(h, 0, c, sc, M, b, yp, N, None, ws.numel(), st) == 1
+    assert lib.trdq_linear_splitk(h, 0, c, sc, M, b, yp, N, wp, 16, st) == 8
+    assert lib.trdq_linear_asym(h, 0, c, sc, z + 2, M, b, yp, N, st) == 3
+    assert lib.trdq_linear_asym(h, 0, c, sc, None, M, b, yp, N, st) == 1
+    torch.cuda.synchronize()
+    assert not y.any().item()                 # none of the refused calls launched anything
+    # M = 0 is a valid empty call everywhere, and an odd but 2-byte aligned bias address is accepted
+    all_equal(calls(M=0), 0)
+    bias_odd = torch.zeros((N + 1,), dtype=torch.bfloat16, device="cuda")
+    bias_odd[1:] = bias
+    expected = trdq.trdq_linear(wts, 0, codes, scales, bias)
+    assert lib.trdq_linear_splitk_static(h, 0, c, sc, M, bias_odd.data_ptr() + 2, yp, N, st) == 0
+    assert torch.equal(y, expected)
+    assert trdq.trdq_device_status() == 0

@@ -85,6 +85,11 @@ def test_host_side_validation_needs_no_device(lib):
     assert lib.trdq_rotate_quantize(None, 0, None, 0, 0, None, None, None) == 1
     assert lib.trdq_linear(None, 0, None, None, 0, None, None, 0, None) == 1
     assert lib.trdq_weights_info(None, None, None, None, None) == 1
+    # the split-K entry points (caller workspace / built-in scratch) and the asymmetric one take a null handle the same way
+    assert lib.trdq_linear_splitk(None, 0, None, None, 0, None, None, 0, None, 0, None) == 1
+    assert lib.trdq_linear_splitk_static(None, 0, None, None, 0, None, None, 0, None) == 1
+    assert lib.trdq_linear_splitk_workspace(None, 0, None, None) == 1
+    assert lib.trdq_linear_asym(None, 0, None, None, None, 0, None, None, 0, None) == 1
     assert lib.trdq_rotation_destroy(None) == 0 and lib.trdq_weights_destroy(None) == 0
     import torch
     if not torch.cuda.is_available():

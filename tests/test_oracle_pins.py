@@ -791,3 +791,102 @@ def test_rotate_f32_equals_rotate_on_bf16_values():
     signs = (rng.integers(0, 2, 384) * 2 - 1).astype(np.int8)
     a, _ = O.fused_vectors(signs, rng.uniform(0.5, 2.0, 384).astype(np.float32))
     assert np.array_equal(O.rotate_f32(f32_of(x_bits), a), O.rotate(x_bits, a))
+
+
+# --------------------------------------------------------------------------- #
+# composite entry points used only by the GPU parity tests
+# --------------------------------------------------------------------------- #
+def test_prepare2_w4_closed_form_and_composition():
+    """Weight side of Eq. 9 with 4-bit storage.  A weight row that is a scaled Hadamard row per block becomes a single spike
+    after the first rotation; the permutation moves the spike (to another block), and the second rotation spreads it into a
+    block of equal magnitudes, so every code is +-7 with the sign pattern of one Hadamard column: a closed form that a wrong
+    permutation direction, nibble order or scale stride breaks."""
+    K = 256
+    unit_w = np.full(K, np.float32(2.0 ** -3.5), np.float32)          # weight vector d / Delta * 2^-3.5 = exactly 1.0
+    _, vec1 = O.fused_vectors(np.ones(K, np.int8), unit_w)
+    assert np.all(vec1 == np.float32(1.0))
+    d2 = np.ones(K, np.int8)
+    d2[[5, 130, 131]] = -1
+    vec2 = O.second_vector(d2, K)
+    c2 = np.float32(2.0 ** -3.5)
+    assert np.array_equal(vec2, (d2.astype(np.float32) * c2))
+    # spikes: block 0 gets 3 at local index 9, block 1 gets -5 at local index 70 (after the first rotation)
+    j0, m0, j1, m1 = 9, 3.0, 70, -5.0
+    idx = np.arange(128)
+    h = lambda j: np.array([(-1.0) ** bin(int(i) & j).count("1") for i in idx])
+    w = np.concatenate([h(j0) * m0 / 128.0, h(j1) * m1 / 128.0])[None, :]
+    wb = bf16(w)
+    assert np.array_equal(f32_of(wb).astype(np.float64), w)
+    v1 = O.rotate(wb, vec1)[0]
+    expect_v1 = np.zeros(K); expect_v1[j0] = m0; expect_v1[128 + j1] = m1
+    assert np.array_equal(v1.astype(np.float64), expect_v1)
+    # (vP)[j] = v[perm[j]]: output slot 131 (block 1, local 3) takes the block-0 spike, slot 5 (block 0) takes the block-1 spike
+    perm = np.arange(K, dtype=np.int32)
+    # (a 4-cycle, so that reading the index vector in the other direction gives a different result)
+    perm[131], perm[j0], perm[5], perm[128 + j1] = j0, 5, 128 + j1, 131
+    assert not np.array_equal(perm[perm], np.arange(K))
+    packed, scales = O.prepare2_w4(wb, vec1, perm, vec2)
+    assert packed.shape == (1, K // 2) and scales.shape == (1, 2)
+    # block 0 of the result holds |m1| * c2 everywhere, block 1 holds |m0| * c2
+    a0 = np.float32(abs(m1)) * c2
+    a1 = np.float32(abs(m0)) * c2
+    assert scales[0, 0] == a0 / np.float32(7.0) and scales[0, 1] == a1 / np.float32(7.0)
+    sign0 = np.sign(m1) * d2[5] * h(5)         # column 5 of the Hadamard block
+    sign1 = np.sign(m0) * d2[131] * h(3)       # column 3
+    codes = np.concatenate([7 * sign0, 7 * sign1]).astype(np.int64)
+    expect = ((codes[0::2] & 0xF) | ((codes[1::2] & 0xF) << 4)).astype(np.uint8)   # even k in the low nibble, two's complement
+    assert np.array_equal(packed[0], expect)
+    assert np.array_equal(O.unpack_w4(packed)[0], codes)
+    # on random rows it is the 4-bit quantiser applied to the full transform's rows
+    rng = np.random.default_rng(77)
+    K2, N2 = 384, 10
+    d1, d2r, smooth, permr = _full_setup(K2, 78)
+    _, wv = O.fused_vectors(d1, smooth)
+    v2 = O.second_vector(d2r, K2)
+    wb2 = bf16(rng.standard_normal((N2, K2)) * 0.02)
+    p_a, s_a = O.prepare2_w4(wb2, wv, permr, v2)
+    p_b, s_b = O.quantize_w4_rows(O.rotate2(wb2, wv, permr, v2))
+    assert np.array_equal(p_a, p_b) and np.array_equal(s_a, s_b)
+    # and not the single-rotation path's result (the permutation and second rotation do something)
+    p_c, _ = O.prepare_w4(wb2, wv)
+    assert not np.array_equal(p_a, p_c)
+
+
+def test_rotate_quantize_asym_ramp_and_composition():
+    """Eq. 1-3 applied to the rotated token (Eq. 10's G_t): input rows whose rotation is a known ramp."""
+    K = 256
+    signs = np.ones(K, np.int8)
+    signs[[0, 2, 133]] = -1
+    act, _ = O.fused_vectors(signs, np.full(K, identity_vec_smooth(), np.float32))
+    assert np.array_equal(act, signs.astype(np.float32))
+    # rotated row: block 0 = 0, 2, .., 254, block 1 = 1, 3, .., 255.  The inverse transform of a ramp 2 i + c is
+    # (127 + c) at index 0 and -2^b at index 2^b (the normalisation is folded into the unit vector above).
+    def block(c):
+        x = np.zeros(128)
+        x[0] = 127.0 + c
+        for b in range(7):
+            x[1 << b] = -(2.0 ** b)
+        return x
+    for shift, z_expect in ((0.0, 0), (-100.0, 100)):
+        x = np.concatenate([block(0.0 + shift), block(1.0 + shift)]) * signs     # the sign diagonal is undone by the vector
+        xb = bf16(x[None, :])
+        assert np.array_equal(f32_of(xb).astype(np.float64)[0], x)
+        v = O.rotate(xb, act)[0]
+        ramp = np.concatenate([2.0 * np.arange(128), 2.0 * np.arange(128) + 1.0]) + shift
+        assert np.array_equal(v.astype(np.float64), ramp)
+        q, s, z = O.rotate_quantize_asym(xb, act)
+        assert q.dtype == np.uint8 and s[0] == np.float32(1.0) and z[0] == z_expect
+        assert np.array_equal(q[0].astype(np.float64), ramp - shift)
+    # on random rows: the asymmetric quantiser applied to the rotated rows, and it depends on the vector
+    rng = np.random.default_rng(79)
+    K2, M2 = 384, 9
+    d = (rng.integers(0, 2, K2) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.25, 4.0, K2).astype(np.float32)
+    a2, _ = O.fused_vectors(d, smooth)
+    xb2 = bf16(rng.standard_normal((M2, K2)) + 0.7)
+    q_a, s_a, z_a = O.rotate_quantize_asym(xb2, a2)
+    q_b, s_b, z_b = O.quantize_rows_asym(O.rotate(xb2, a2))
+    assert np.array_equal(q_a, q_b) and np.array_equal(s_a, s_b) and np.array_equal(z_a, z_b)
+    a3, _ = O.fused_vectors(d, None)
+    q_c, _, _ = O.rotate_quantize_asym(xb2, a3)
+    assert not np.array_equal(q_a, q_c)

@@ -56,7 +56,7 @@ def check_output(y_gpu: np.ndarray, y_ref: np.ndarray, max_ulp: float = 2.0, rel
     return float(l2), float(ulps.max())
 
 
-def check_codes_with_tolerance(codes: np.ndarray, scales: np.ndarray, v_ref: np.ndarray, tol_v: np.ndarray, max_fraction: float = 2e-3):
+def check_codes_with_tolerance(codes: np.ndarray, scales: np.ndarray, v_ref: np.ndarray, tol_v: np.ndarray, max_fraction: float = 1e-4):
     """Codes and scales of a path whose pre-quantization values v agree with the oracle's only up to tol_v (elementwise,
     absolute): scales may differ by the tolerance at the row maximum (over 127), a code may differ by one step and only
     where the oracle's value before rounding lies within the propagated tolerance of a .5 boundary.  Returns the count."""
