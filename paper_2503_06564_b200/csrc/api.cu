@@ -459,8 +459,8 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
                                                    static_cast<cudaStream_t>(stream));
     return e2 == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
   }
-  if (rotate_quantize_prefers_tma(M, rot->K))
-    return launch_rotate_quantize_tma(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream));
+  if (rotate_quantize_prefers_team(M, rot->K))
+    return launch_rotate_quantize_team(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream));
   const cudaError_t e = launch_rotate_quantize(X_bf16, ldx, M, rot->K, vec, 0, codes, scales, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
 }

@@ -78,11 +78,10 @@ cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, i
 cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec1, const int32_t* perm,
                                     const float* vec2, int mode, void* codes, float* scales, cudaStream_t stream);
 
-// rotate_quantize_tma.cu: per-row int8 path for rows of at most 36 blocks (TMA-staged, one thread per block)
-int rotate_quantize_tma_rows(int32_t K);  // rows per tile, 0 if K is too wide for this kernel
-bool rotate_quantize_prefers_tma(int32_t M, int32_t K);
-trdq_status launch_rotate_quantize_tma(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
-                                       float* scales, cudaStream_t stream);
+// rotate_quantize_team.cu: per-row int8 path, TMA-staged, one thread per block, independent teams of warps per CTA
+bool rotate_quantize_prefers_team(int32_t M, int32_t K);
+trdq_status launch_rotate_quantize_team(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int8_t* codes,
+                                        float* scales, cudaStream_t stream);
 
 // norm_rotate_quantize.cu: LayerNorm + per-sample modulation in front of the rotation (K <= 8192)
 cudaError_t launch_norm_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, const void* shift_bf16,
