@@ -30,8 +30,7 @@ UNIT = "TOPS"
 # DRAM traffic per unit of algorithmic work, from the Nsight Compute captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch); None once a kernel has changed since its capture.
 GEMM_PAIR_DRAM_BYTES_PER_OP = 123.3e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
-RQ_TMA_DRAM_BYTES_PER_ALG_BYTE = 191.7 / 226.6      # rotate_quantize_tma_kernel, M = 65536, K = 1152
-RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE = 20.8 / 31.1       # rotate_quantize_rows_kernel, M = 9000, K = 1152
+RQ_TEAM_DRAM_BYTES_PER_ALG_BYTE = None              # rotate_quantize_team_kernel: set from its capture under profiles/
 INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -197,36 +196,51 @@ def time_region(fn, steps: int):
     return e0.elapsed_time(e1)
 
 
-def kernel_pass_ms(layers, wl, which: str, reps: int):
-    """Average time (ms) of one step's launches of ONE kernel kind, replayed from a CUDA graph so the
-    launches are back to back.  which = 'rq' (rotate + quantize) or 'gemm' (GEMM + epilogue)."""
-    import torch
-    from paper_2503_06564_b200 import trdq
-    t = int(wl.timesteps()[0])
-    keep = layers._keep
+class KernelPass:
+    """One step's launches of ONE kernel kind (rotate + quantize, or GEMM + epilogue) captured in a CUDA graph, so that
+    the launches run back to back on the device."""
 
-    def issue():
-        for (rot, w, x, codes, scales, bias, y), ws in zip(keep, layers._extra):
-            if which == "rq" and ws is not None:
-                trdq.trdq_rotate_dense_quantize(rot, t, x, codes, scales, ws)
-            elif which == "rq":
-                trdq.trdq_rotate_quantize(rot, t, x, codes, scales)
-            else:
-                trdq.trdq_linear(w, t, codes, scales, bias, y)
+    def __init__(self, layers, wl, which: str):
+        import torch
+        from paper_2503_06564_b200 import trdq
+        t = int(wl.timesteps()[0])
+        keep = layers._keep
 
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        issue()
-    torch.cuda.current_stream().wait_stream(side)
-    torch.cuda.synchronize()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, capture_error_mode="thread_local"):
-        issue()
-    for _ in range(3):
-        graph.replay()
-    ms = time_region(lambda i: graph.replay(), reps)
-    return ms / reps
+        def issue():
+            for (rot, w, x, codes, scales, bias, y), ws in zip(keep, layers._extra):
+                if which == "rq" and ws is not None:
+                    trdq.trdq_rotate_dense_quantize(rot, t, x, codes, scales, ws)
+                elif which == "rq":
+                    trdq.trdq_rotate_quantize(rot, t, x, codes, scales)
+                else:
+                    trdq.trdq_linear(w, t, codes, scales, bias, y)
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            issue()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph, capture_error_mode="thread_local"):
+            issue()
+        for _ in range(3):
+            self.graph.replay()
+        torch.cuda.synchronize()
+
+    def ms(self, reps: int = 0, min_seconds: float = 0.0):
+        """(ms per pass, seconds timed): `reps` passes, or as many as fill `min_seconds`; a tenth of them untimed first."""
+        once = time_region(lambda i: self.graph.replay(), 3) / 3
+        if min_seconds > 0.0:
+            reps = max(reps, int(np.ceil(1.1 * min_seconds * 1e3 / max(once, 1e-6))))
+        reps = max(reps, 3)
+        for _ in range(max(3, reps // 10)):
+            self.graph.replay()
+        total = time_region(lambda i: self.graph.replay(), reps)
+        if min_seconds > 0.0 and total * 1e-3 < min_seconds:      # the first estimate was taken at other clocks
+            reps = int(np.ceil(reps * 1.2 * min_seconds / (total * 1e-3)))
+            total = time_region(lambda i: self.graph.replay(), reps)
+        return total / reps, total * 1e-3
 
 
 # ------------------------------------------------------------------------------------------
@@ -269,27 +283,6 @@ def block_ops(wl: WL.Workload, rows: int) -> float:
     return sum(2.0 * min(rows, l.M or wl.M) * l.N * l.K for l in wl.layers + wl.extra_layers)
 
 
-def cpu_baseline(wl: WL.Workload, budget_s: float = 20.0):
-    """The oracle as it stands on this host's cores, on a bounded sample: whole blocks of the step (or, for the large
-    workloads, one block with as many token rows as fit the time budget, calibrated on 32 rows first)."""
-    from oracle import trdq_oracle as O
-    cal_rows = 32
-    cal = oracle_block_inputs(wl, cal_rows)
-    oracle_block_seconds(wl, cal)                                  # warm the thread pool
-    per_row = oracle_block_seconds(wl, cal) / cal_rows
-    rows = int(max(cal_rows, min(wl.M, budget_s / max(per_row, 1e-9))))
-    items = oracle_block_inputs(wl, rows)
-    sec = oracle_block_seconds(wl, items)
-    # when a whole block takes only a second or two, go through more of the step's (identically shaped) blocks: 10 - 30 s in all
-    blocks_done = 1
-    while sec < 10.0 and blocks_done < wl.blocks:
-        sec += oracle_block_seconds(wl, items)
-        blocks_done += 1
-    tops = blocks_done * block_ops(wl, rows) / sec / 1e12
-    return {"value": tops, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-            "sample": f"{blocks_done} of {wl.blocks} blocks ({len(items)} linears each), first {rows} of {wl.M} token rows, {sec:.2f} s"}
-
-
 def run_reference(args, wl: WL.Workload):
     """`--impl reference`: the CPU oracle on this host, each step a bounded sample of the workload."""
     from oracle import trdq_oracle as O
@@ -325,10 +318,191 @@ def run_reference(args, wl: WL.Workload):
 # ------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------
+NOMINAL_INT8_TOPS = 4500.0     # dense INT8, public figure for the part
+NOMINAL_HBM_GBS = 8000.0
+
+
+def peak_for(peaks, seconds: float):
+    """Tensor-core denominator by the length of the timed region: the burst figure for a region under a second, the
+    sustained (power-capped) one for a region of two seconds or more; in between, the burst figure (the harder one)."""
+    if seconds >= 2.0:
+        return peaks["bf16_tflops_sustained"] * INT8_OVER_BF16, "sustained"
+    return peaks["bf16_tflops"] * INT8_OVER_BF16, "burst"
+
+
+def kernel_names(wl: WL.Workload):
+    """Kernel the library runs per layer (asked from the library itself), and for each stage the kernel that does
+    most of the work of a step."""
+    from paper_2503_06564_b200 import trdq
+    rq, gemm, per_layer = {}, {}, []
+    for layer in wl.layers + wl.extra_layers:
+        m = layer.M or wl.M
+        a = trdq.trdq_kernel_choice(0, m, layer.K)
+        b = trdq.trdq_kernel_choice(1, m, layer.K, layer.N, wl.wbits)
+        per_layer.append({"layer": layer.name, "M": m, "K": layer.K, "N": layer.N, "rotate_quantize": a, "linear": b})
+        rq[a] = rq.get(a, 0.0) + m * (3.0 * layer.K + 4.0)
+        b0 = b.split("<")[0]
+        gemm[b0] = gemm.get(b0, 0.0) + 2.0 * m * layer.N * layer.K
+    return max(rq, key=rq.get), max(gemm, key=gemm.get), per_layer
+
+
+def roofline_entries(wl, peaks, ops, ms_gemm, sec_gemm, ms_rq, sec_rq, dense=False):
+    rq_kernel, gemm_kernel, per_layer = kernel_names(wl)
+    if dense:
+        rq_kernel = "rotate_dense_amax_kernel+rotate_dense_quantize_kernel"
+    int8_peak, which = peak_for(peaks, sec_gemm)
+    gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
+    rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
+    n_ops = len(wl.layers + wl.extra_layers) * wl.blocks
+    gemm = {"kernel": gemm_kernel, "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOPS",
+            "frac": gemm_tops / int8_peak, "frac_nominal": gemm_tops / NOMINAL_INT8_TOPS, "seconds_timed": sec_gemm,
+            "peak_source": f"{peaks['_source']} {which} bf16 {int8_peak / INT8_OVER_BF16:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16); "
+                           f"nominal {NOMINAL_INT8_TOPS:g} TOPS",
+            "traffic": (GEMM_PAIR_DRAM_BYTES_PER_OP * ops / n_ops) if gemm_kernel == "gemm_w8a8_pair_kernel" else None,
+            "traffic_note": "bytes per launch, scaled by operations from the capture in profiles/gemm_w8a8_pair_*.txt to an average launch of this workload"}
+    rq = {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+          "frac": rq_gbs / peaks["hbm_gbs"], "frac_nominal": rq_gbs / NOMINAL_HBM_GBS, "seconds_timed": sec_rq,
+          "peak_source": f"{peaks['_source']} copy rate; nominal {NOMINAL_HBM_GBS:g} GB/s",
+          "traffic": RQ_TEAM_DRAM_BYTES_PER_ALG_BYTE * step_rq_bytes(wl) / n_ops
+          if (rq_kernel == "rotate_quantize_team_kernel" and RQ_TEAM_DRAM_BYTES_PER_ALG_BYTE) else None,
+          "traffic_note": "bytes per launch, scaled by algorithmic bytes from the capture in profiles/rotate_quantize_team_*.txt"}
+    return gemm, rq, per_layer
+
+
+class DeviceRun:
+    """A workload resident on the device with its per-group CUDA graphs."""
+
+    def __init__(self, wl, args, rank):
+        import torch
+        from paper_2503_06564_b200 import trdq
+        self.wl = wl
+        self.layers = build_device_workload(wl, seed=1234 + rank, blocks=wl.blocks, rotation=args.rotation)
+        self.ts = wl.timesteps()
+        layers, ts = self.layers, self.ts
+        for i in range(3):
+            trdq.trdq_run_layers(layers, int(ts[i % len(ts)]))
+        torch.cuda.synchronize()
+        assert trdq.trdq_device_status() == 0
+        # One CUDA graph per time-step group (the kernels of a step depend on t only through its group: a group switch
+        # is a switch of graph); the step of the sampling loop replays the graph of its group.
+        self.graphs = {}
+        if not args.no_graph:
+            side = torch.cuda.Stream()
+            for t in ts:
+                g = trdq.trdq_find_group(wl.t_bounds, int(t))
+                if g in self.graphs:
+                    continue
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    trdq.trdq_run_layers(layers, int(t))
+                torch.cuda.current_stream().wait_stream(side)
+                torch.cuda.synchronize()
+                self.graphs[g] = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(self.graphs[g], capture_error_mode="thread_local"):
+                    trdq.trdq_run_layers(layers, int(t))
+            self.groups_of_steps = [trdq.trdq_find_group(wl.t_bounds, int(t)) for t in ts]
+
+    def step(self, i):
+        from paper_2503_06564_b200 import trdq
+        if self.graphs:
+            self.graphs[self.groups_of_steps[i % len(self.ts)]].replay()
+        else:
+            trdq.trdq_run_layers(self.layers, int(self.ts[i % len(self.ts)]))
+
+
+def measure_side_workload(wl, args, rank, peaks):
+    """Short passes of a workload other than the headline one: step time, both kernel classes, clocks."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    run = DeviceRun(wl, args, rank)
+    for i in range(3):
+        run.step(i)
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    steps = max(5, min(args.steps, 20)) if wl.index != 0 else 200
+    ms = time_region(run.step, steps) / steps
+    ms_rq, sec_rq = KernelPass(run.layers, wl, "rq").ms(reps=steps)
+    ms_gemm, sec_gemm = KernelPass(run.layers, wl, "gemm").ms(reps=steps)
+    clocks = sampler.stop()
+    assert trdq.trdq_device_status() == 0
+    ops = step_ops(wl)
+    gemm, rq, _ = roofline_entries(wl, peaks, ops, ms_gemm, sec_gemm, ms_rq, sec_rq)
+    for d in (gemm, rq):
+        for k in ("traffic", "traffic_note", "peak_source", "bound", "unit"):
+            d.pop(k, None)
+    out = {"workload": wl.name, "M": wl.M, "wbits": wl.wbits, "steps": steps, "ms_per_step": ms, "us_per_dit_step": ms * 1e3,
+           "tops": ops / (ms * 1e-3) / 1e12, "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
+           "gemm": gemm, "rotate_quantize": rq, "clocks": clocks}
+    del run
+    torch.cuda.empty_cache()
+    return out
+
+
+def gpu_parity_and_cpu_baseline(wl: WL.Workload, budget_s: float = 20.0):
+    """The cpu_baseline leg: the oracle as it stands, timed on this host's cores on a bounded sample of the workload's
+    own seeded inputs (whole blocks of the step, or one block with as many token rows as fit the budget) - and, since it
+    has then computed those rows, the same inputs are run through the library in the launch configuration the benchmark
+    times (trdq_run_layers) and compared: activation codes and scales bit for bit, outputs in bf16 steps."""
+    import torch
+    from oracle import trdq_oracle as O
+    from paper_2503_06564_b200 import trdq
+    cal_rows = 32
+    cal = oracle_block_inputs(wl, cal_rows)
+    oracle_block_seconds(wl, cal)                                  # warm the thread pool
+    per_row = oracle_block_seconds(wl, cal) / cal_rows
+    rows = int(max(cal_rows, min(wl.M, budget_s / max(per_row, 1e-9))))
+    items = oracle_block_inputs(wl, rows)
+    t = int(wl.timesteps()[0])
+    t0 = time.perf_counter()
+    refs = []
+    for inp, act, qw, sw, m in items:
+        q, sx = O.rotate_quantize(inp.x, act)
+        idx = np.arange(m)
+        y = O.linear_w8_rows(q, sx, qw, sw, inp.bias, idx) if wl.wbits == 8 else O.linear_w4_rows(q, sx, qw, sw, inp.bias, idx)
+        refs.append((q, sx, y))
+    sec = time.perf_counter() - t0
+    blocks_done = 1
+    while sec < 10.0 and blocks_done < wl.blocks:
+        sec += oracle_block_seconds(wl, items)
+        blocks_done += 1
+    tops = blocks_done * block_ops(wl, rows) / sec / 1e12
+    baseline = {"value": tops, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+                "sample": f"{blocks_done} of {wl.blocks} blocks ({len(items)} linears each), first {rows} of {wl.M} token rows, {sec:.2f} s"}
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+    layers, outs = trdq.LayerList(), []
+    for inp, act, qw, sw, m in items:
+        rot = trdq.Rotation(inp.layer.K, inp.t_bounds, inp.signs, inp.smooth)
+        wts = trdq.trdq_prepare_weights(rot, dev(inp.w), wl.wbits)
+        codes = torch.empty((m, inp.layer.K), dtype=torch.int8, device="cuda")
+        scales = torch.empty((m,), dtype=torch.float32, device="cuda")
+        y = torch.empty((m, inp.layer.N), dtype=torch.bfloat16, device="cuda")
+        layers.add(rot, wts, dev(inp.x), codes, scales, dev(inp.bias), y)
+        outs.append((codes, scales, y))
+    trdq.trdq_run_layers(layers, t)
+    torch.cuda.synchronize()
+    codes_equal, scales_equal, max_steps, worst_l2, n_out = True, True, 0.0, 0.0, 0
+    for (q, sx, y_ref), (codes, scales, y) in zip(refs, outs):
+        codes_equal &= bool(np.array_equal(codes.cpu().numpy(), q))
+        scales_equal &= bool(np.array_equal(scales.cpu().numpy(), sx))
+        y_gpu = WL.bf16_bits_to_f32(y.view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+        err = np.abs(y_gpu - y_ref)
+        _, e = np.frexp(np.abs(y_ref).astype(np.float64))
+        max_steps = max(max_steps, float((err / np.ldexp(1.0, np.maximum(e - 8, -133))).max()))
+        worst_l2 = max(worst_l2, float(np.sqrt((err ** 2).sum() / max((y_ref.astype(np.float64) ** 2).sum(), 1e-300))))
+        n_out += y_ref.size
+    parity = {"against": "oracle", "launch": "trdq_run_layers", "linears": len(items), "rows": rows, "outputs": n_out,
+              "codes_bit_exact": codes_equal, "scales_bit_exact": scales_equal, "max_bf16_steps": max_steps, "rel_l2": worst_l2,
+              "ok": bool(codes_equal and scales_equal and max_steps <= 2.0 and worst_l2 <= 2e-3)}
+    return baseline, parity
+
+
 def run_ours(args, wl: WL.Workload):
     import torch
     import torch.distributed as dist
-    from paper_2503_06564_b200 import build as lib_build, multirank, trdq
+    from paper_2503_06564_b200 import build as lib_build, microbench, multirank, trdq
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -341,46 +515,13 @@ def run_ours(args, wl: WL.Workload):
     if world > 1:
         dist.barrier()
     trdq.lib()                                   # fails loudly if the CUDA library is missing
+    peaks = load_peaks()
 
     # weak scaling: every rank runs the whole workload on its own batch (rows are independent; no collective)
-    layers = build_device_workload(wl, seed=1234 + rank, blocks=wl.blocks, rotation=args.rotation)
-    ts = wl.timesteps()
-    n_ops = len(layers)
-
-    def step_direct(i):
-        trdq.trdq_run_layers(layers, int(ts[i % len(ts)]))
-
+    run = DeviceRun(wl, args, rank)
+    layers, ts, n_ops = run.layers, run.ts, len(run.layers)
+    step = run.step
     for i in range(max(args.warmup, 3)):
-        step_direct(i)
-    torch.cuda.synchronize()
-    assert trdq.trdq_device_status() == 0
-
-    # One CUDA graph per time-step group (the kernels of a step depend on t only through its group: a group switch is a
-    # switch of graph); the step of the sampling loop replays the graph of its group.
-    graphs = {}
-    if not args.no_graph:
-        side = torch.cuda.Stream()
-        for t in ts:
-            g = trdq.trdq_find_group(wl.t_bounds, int(t))
-            if g in graphs:
-                continue
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                trdq.trdq_run_layers(layers, int(t))
-            torch.cuda.current_stream().wait_stream(side)
-            torch.cuda.synchronize()
-            graphs[g] = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graphs[g], capture_error_mode="thread_local"):
-                trdq.trdq_run_layers(layers, int(t))
-        groups_of_steps = [trdq.trdq_find_group(wl.t_bounds, int(t)) for t in ts]
-
-    def step(i):
-        if graphs:
-            graphs[groups_of_steps[i % len(ts)]].replay()
-        else:
-            step_direct(i)
-
-    for i in range(3):
         step(i)
     torch.cuda.synchronize()
 
@@ -392,25 +533,49 @@ def run_ours(args, wl: WL.Workload):
     ms = multirank.max_over_ranks(ms, device="cuda")
     if world > 1:
         dist.barrier()
-    # per-kernel passes (same buffers, launches back to back from a CUDA graph)
-    reps = max(3, min(args.steps, 20))
-    ms_rq = kernel_pass_ms(layers, wl, "rq", reps)
-    ms_gemm = kernel_pass_ms(layers, wl, "gemm", reps)
     clocks = sampler.stop()
-    assert trdq.trdq_device_status() == 0, "a bounded device-side wait expired during the benchmark"
-
     ops = step_ops(wl)
     ms_per_step = ms / args.steps
     value = world * ops / (ms_per_step * 1e-3) / 1e12
 
-    # end to end through the public call with host buffers: H2D of every X, the step, D2H of every Y
+    # Per-kernel passes on the same buffers, launches back to back from a CUDA graph: once for at least two seconds (the
+    # part settles under its power cap: compared with the sustained peak) and once briefly (compared with the burst peak).
+    dense = args.rotation == "dense"
+    long_s = 0.0 if args.quick else 2.0
+    sampler2 = ClockSampler(local_rank)
+    sampler2.start()
+    gemm_pass, rq_pass = KernelPass(layers, wl, "gemm"), KernelPass(layers, wl, "rq")
+    ms_gemm, sec_gemm = gemm_pass.ms(reps=3, min_seconds=long_s)
+    ms_rq, sec_rq = rq_pass.ms(reps=3, min_seconds=long_s)
+    reps_long = max(args.steps, int(np.ceil(long_s * 1e3 / ms_per_step)))
+    ms_sustained = time_region(step, reps_long) / reps_long
+    clocks_sustained = sampler2.stop()
+    # brief passes (a few tenths of a second each, after a pause): compared with the burst peak
+    time.sleep(0.0 if args.quick else 1.0)
+    ms_gemm_b, sec_gemm_b = gemm_pass.ms(min_seconds=0.25)
+    time.sleep(0.0 if args.quick else 1.0)
+    ms_rq_b, sec_rq_b = rq_pass.ms(min_seconds=0.25)
+    assert trdq.trdq_device_status() == 0, "a bounded device-side wait expired during the benchmark"
+    roof_gemm, roof_rq, per_layer = roofline_entries(wl, peaks, ops, ms_gemm, sec_gemm, ms_rq, sec_rq, dense)
+    burst_gemm, burst_rq, _ = roofline_entries(wl, peaks, ops, ms_gemm_b, sec_gemm_b, ms_rq_b, sec_rq_b, dense)
+    roof_gemm["brief"] = {k: burst_gemm[k] for k in ("achieved", "peak", "frac", "frac_nominal", "seconds_timed", "peak_source")}
+    roof_rq["brief"] = {k: burst_rq[k] for k in ("achieved", "frac", "frac_nominal", "seconds_timed")}
+    ceiling = None
+    if rank == 0 and wl.wbits == 8:
+        c = microbench.mma_ceiling(65536, 5)
+        ceiling = {"kernel": c["kernel"], "tops": c["rate_best"], "what": "back-to-back 256x256x32 int8 MMAs per CTA pair on resident operands"}
+        roof_gemm["frac_of_mma_ceiling"] = roof_gemm["achieved"] / c["rate_best"]
+
+    # end to end through the public call with host buffers: H2D of every X, the step, D2H of every Y.  The pinned host
+    # buffers hold ONE transformer block's tensors and serve every block (the bytes moved are those of the whole step).
     e2e_steps = max(1, min(args.steps, 3))
-    host_x = [torch.empty(k[2].shape, dtype=k[2].dtype).pin_memory() for k in layers._keep]
-    host_y = [torch.empty(k[6].shape, dtype=k[6].dtype).pin_memory() for k in layers._keep]
+    per_block = len(wl.layers + wl.extra_layers)
+    host_x = [torch.empty(k[2].shape, dtype=k[2].dtype).pin_memory() for k in layers._keep[:per_block]]
+    host_y = [torch.empty(k[6].shape, dtype=k[6].dtype).pin_memory() for k in layers._keep[:per_block]]
     for hx, k in zip(host_x, layers._keep):
         hx.copy_(k[2])
-    h2d = sum(h.numel() * h.element_size() for h in host_x)
-    d2h = sum(h.numel() * h.element_size() for h in host_y)
+    h2d = sum(k[2].numel() * k[2].element_size() for k in layers._keep)
+    d2h = sum(k[6].numel() * k[6].element_size() for k in layers._keep)
 
     # Copies and kernels are pipelined layer by layer over three streams (PCIe carries both directions at once): layer i's
     # kernels wait for its input copy, its output copy waits for its kernels; across steps a buffer is not overwritten before
@@ -426,7 +591,8 @@ def run_ours(args, wl: WL.Workload):
         t = int(ts[i % len(ts)])
         s_in.wait_stream(s_main)        # buffers written before this step (warm-up, the step before) are complete
         s_out.wait_stream(s_main)
-        for j, (hx, hy, k) in enumerate(zip(host_x, host_y, layers._keep)):
+        for j, k in enumerate(layers._keep):
+            hx, hy = host_x[j % per_block], host_y[j % per_block]
             with torch.cuda.stream(s_in):
                 if not first_e2e[0]:
                     s_in.wait_event(ev_done[j])       # the step before has read X_j
@@ -448,28 +614,8 @@ def run_ours(args, wl: WL.Workload):
     e2e_step(0)
     ms_e2e = time_region(e2e_step, e2e_steps) / e2e_steps
     ms_e2e = multirank.max_over_ranks(ms_e2e, device="cuda")
+    assert trdq.trdq_device_status() == 0
 
-    peaks = load_peaks()
-    in_long_step = True
-    bf16_peak = peaks["bf16_tflops_sustained"] if in_long_step else peaks["bf16_tflops"]
-    int8_peak = bf16_peak * INT8_OVER_BF16
-    gemm_kernel = "gemm_w4a8_kernel" if wl.wbits == 4 else ("gemm_w8a8_pair_kernel" if wl.M >= 2048 else "gemm_w8a8_kernel")
-    # which rotate + quantize kernel the library picks per layer (rows of <= 36 blocks and >= 6 rounds of one tile per SM
-    # go to the TMA-staged kernel), and the kernel that moves most of the step's bytes
-    sms = torch.cuda.get_device_properties(0).multi_processor_count
-    rq_bytes = {"rotate_quantize_tma_kernel": 0.0, "rotate_quantize_rows_kernel": 0.0}
-    for layer in wl.layers + wl.extra_layers:
-        m, nb = (layer.M or wl.M), layer.K // 128
-        r = (288 // nb) // 8 * 8 if nb <= 36 else 0
-        tma = r > 0 and (m + r - 1) // r >= 6 * sms
-        rq_bytes["rotate_quantize_tma_kernel" if tma else "rotate_quantize_rows_kernel"] += m * (3.0 * layer.K + 4.0)
-    rq_kernel = max(rq_bytes, key=rq_bytes.get)
-    rq_traffic_ratio = RQ_TMA_DRAM_BYTES_PER_ALG_BYTE if rq_kernel == "rotate_quantize_tma_kernel" else RQ_ROWS_DRAM_BYTES_PER_ALG_BYTE
-    dense = args.rotation == "dense"
-    if dense:
-        rq_kernel, rq_traffic_ratio = "rotate_dense_amax_kernel+rotate_dense_quantize_kernel", None
-    gemm_tops = ops / (ms_gemm * 1e-3) / 1e12
-    rq_gbs = step_rq_bytes(wl) / (ms_rq * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -477,30 +623,30 @@ def run_ours(args, wl: WL.Workload):
         "config": {"workload": wl.name, "M": wl.M, "blocks": wl.blocks, "linears_per_step": n_ops, "groups": wl.num_groups,
                    "sampling_steps": wl.steps, "wbits": wl.wbits, "parallelism": f"replicas x{world} (rows independent)",
                    "rotation": args.rotation, "launch": "host" if args.no_graph else "one CUDA graph per time-step group",
-
                    "l2": "inputs larger than L2: every linear has its own X, codes, Y and weights"},
         "us_per_dit_step": ms_per_step * 1e3,
-        "rotate_quantize_gbs": rq_gbs,
-        "gemm_tops": gemm_tops,
+        "rotate_quantize_gbs": roof_rq["achieved"],
+        "gemm_tops": roof_gemm["achieved"],
         "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
-        "roofline": {"kernel": gemm_kernel, "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
-                     "unit": "TOPS", "frac": gemm_tops / int8_peak,
-                     "traffic": (GEMM_PAIR_DRAM_BYTES_PER_OP * ops / n_ops) if gemm_kernel == "gemm_w8a8_pair_kernel" else None,
-                     "traffic_note": "bytes per launch: capture at M=16384,K=1152,N=4608 scaled by the ops of an average launch of this workload",
-                     "peak_source": f"{peaks['_source']} sustained bf16 {bf16_peak:.1f} TFLOP/s x {INT8_OVER_BF16:g} (nominal int8:bf16)"},
-        "roofline_rotate_quantize": {"kernel": rq_kernel, "bound": "hbm", "achieved": rq_gbs,
-                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
-                                     "traffic": None if rq_traffic_ratio is None else rq_traffic_ratio * step_rq_bytes(wl) / n_ops,
-                                     "traffic_note": "bytes per launch: capture of this kernel (TMA: M=65536,K=1152; rows: M=9000,K=1152) scaled by algorithmic bytes",
-                                     "peak_source": peaks["_source"]},
+        "sustained": {"ms_per_step": ms_sustained, "steps": reps_long, "tops": ops / (ms_sustained * 1e-3) / 1e12,
+                      "clocks": clocks_sustained, "what": "the same step loop run for at least two seconds, after the per-kernel passes"},
+        "roofline": roof_gemm,
+        "roofline_rotate_quantize": roof_rq,
+        "mma_ceiling": ceiling,
+        "kernels_per_layer": per_layer,
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},
         "gpu_launches": (3 if dense else 2) * n_ops * args.steps,
         "clocks": clocks,
     }
+    del run, layers, gemm_pass, rq_pass, host_x, host_y, step
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not dense:
+        if not args.no_per_workload:
+            line["per_workload"] = [measure_side_workload(w2, args, rank, peaks) for w2 in WL.WORKLOADS if w2.index != wl.index]
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"], line["parity"] = gpu_parity_and_cpu_baseline(wl)
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline and not dense:
-            line["cpu_baseline"] = cpu_baseline(wl)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -510,16 +656,27 @@ def run_ours(args, wl: WL.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, help="index into the workload list (1 = DiT-XL/2 256px, M = 4096)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", type=int, default=3,
+                    help="index into the workload list; default 3 = PixArt-style 1024 px, M = 32768 plus cross-attention, the largest "
+                         "single-GPU 8-bit configuration (1 = DiT-XL/2 256 px, 2 = 512 px, 4 = video DiT W4A8, 0 = single layer)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle leg (CPU baseline and the parity check that rides on it)")
+    ap.add_argument("--no-per-workload", action="store_true", help="skip the short passes over the other workloads")
+    ap.add_argument("--quick", action="store_true", help="no two-second passes (development runs)")
     ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host instead of replaying one CUDA graph per time-step group")
     ap.add_argument("--rotation", default="hadamard", choices=["hadamard", "dense"],
                     help="hadamard: the headline path; dense: dense 128 x 128 blocks on the tensor cores (Eq. 6-8), no CPU baseline")
     args = ap.parse_args()
     wl = WL.WORKLOADS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for several GPUs outside a launcher: start one process per GPU here (rank 0 prints the line)
+        from paper_2503_06564_b200 import multirank
+        rc, out = multirank.spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+        sys.stdout.write(out)
+        sys.stdout.flush()
+        sys.exit(rc)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

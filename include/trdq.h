@@ -325,6 +325,22 @@ trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes,
  * receives the raw bits. */
 trdq_status trdq_device_status(uint32_t* word);
 
+/* Reports which kernel a call would run on the current device, for benchmark and profile reports (the paper has no
+ * counterpart).  stage 0: trdq_rotate_quantize on M rows of K channels (N, wbits ignored); stage 1: trdq_linear on M rows
+ * against [N, K] weights of `wbits` bits.  `name` (host, at least 48 bytes, `name_bytes` its size) receives a
+ * NUL-terminated kernel name such as "gemm_w8a8_pair_kernel<256>".  The answer comes from the same functions the
+ * launchers use.  TRDQ_ERR_CUDA without a device: the choice depends on its SM count. */
+trdq_status trdq_kernel_choice(int32_t stage, int32_t M, int32_t K, int32_t N, int32_t wbits, char* name, int32_t name_bytes);
+
+/* Measurement aid (the paper has no counterpart): runs the tensor pipe by itself.  Every resident CTA pair issues
+ * `mmas_per_cluster` (8 ... 2^22) back-to-back tcgen05.mma cta_group::2 kind::i8 of shape 256 x 256 x 32 on constant
+ * operands that already sit in shared memory: no loads, no epilogue, nothing is written to global memory.
+ * `*clusters` (host) receives the number of CTA pairs launched, so one launch performs
+ *     clusters * mmas_per_cluster * 2 * 256 * 256 * 32   integer operations;
+ * the caller times the launch on `stream`.  The rate is the ceiling of the INT8 GEMM at the clocks the device runs at.
+ * The wait for completion is bounded like every other one (trdq_device_status reports an expiry). */
+trdq_status trdq_measure_mma_ceiling(int32_t mmas_per_cluster, int32_t* clusters, void* stream);
+
 /* Exercises the bounded wait on purpose: launches one warp that waits on a memory barrier nothing will ever
  * signal.  The wait expires after 20 ms, sets bit 31 of the status word and the kernel ends normally; the next
  * trdq_device_status returns TRDQ_ERR_TIMEOUT with that bit and clears it, and the device stays fully usable.

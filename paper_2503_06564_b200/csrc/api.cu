@@ -3,6 +3,7 @@
 // happens here except the fused per-channel vectors, which are formed once per group.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstring>
 #include <new>
 
@@ -652,6 +653,27 @@ trdq_status trdq_run_layers(const trdq_layer_op* ops, int32_t count, int32_t t, 
     if (st != TRDQ_OK) return st;
   }
   return TRDQ_OK;
+}
+
+trdq_status trdq_kernel_choice(int32_t stage, int32_t M, int32_t K, int32_t N, int32_t wbits, char* name, int32_t name_bytes) {
+  if (!name) return TRDQ_ERR_NULL;
+  if (name_bytes < 48 || M <= 0 || K <= 0 || K % TRDQ_BLOCK != 0) return TRDQ_ERR_SHAPE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;  // the choice depends on the device (SM count, resident clusters)
+  if (stage == 0) {
+    describe_rotate_quantize_kernel(M, K, name, static_cast<size_t>(name_bytes));
+    return TRDQ_OK;
+  }
+  if (stage != 1 || N <= 0) return TRDQ_ERR_SHAPE;
+  if (wbits != 8 && wbits != 4) return TRDQ_ERR_WBITS;
+  describe_gemm_kernel(M, K, N, wbits, name, static_cast<size_t>(name_bytes));
+  return TRDQ_OK;
+}
+
+trdq_status trdq_measure_mma_ceiling(int32_t mmas_per_cluster, int32_t* clusters, void* stream) {
+  if (!clusters) return TRDQ_ERR_NULL;
+  if (mmas_per_cluster < 8 || mmas_per_cluster > (1 << 22)) return TRDQ_ERR_SHAPE;
+  return launch_mma_ceiling(mmas_per_cluster, clusters, static_cast<cudaStream_t>(stream));
 }
 
 trdq_status trdq_selftest_wait_expiry(void* stream) {

@@ -18,6 +18,7 @@
 // once for both.  Every wait is bounded (see BoundedWaiter).
 #include <cuda_bf16.h>
 
+#include <cstdio>
 #include <cstdlib>
 
 #include "epilogue.cuh"
@@ -349,15 +350,38 @@ int choose_tile_n(int64_t tiles_m, int N, int sms) {
 
 }  // namespace
 
-static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, int mode,
-                                       const int32_t* const zp[2], cudaStream_t stream, int act = 0) {
-  const bool raw_i32 = mode == 1;
-  // Large problems go to the CTA-pair kernel (two SMs per 256-row tile, a third less operand traffic per SM).
-  static const int pair_min_rows = [] {
+// Row count from which the CTA-pair kernel is used (two SMs per 256-row tile, a third less operand traffic per SM).
+static int pair_min_rows() {
+  static const int rows = [] {
     const char* e = getenv("TRDQ_PAIR_MIN_M");
     return e ? atoi(e) : 2048;
   }();
-  if (mode == 0 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows) {
+  return rows;
+}
+
+// Name of the kernel trdq_linear runs for M rows against [N, K] weights of `wbits` bits (one row segment).
+void describe_gemm_kernel(int32_t M, int32_t K, int32_t N, int32_t wbits, char* name, size_t cap) {
+  (void)K;
+  if (wbits == 4) {
+    snprintf(name, cap, "gemm_w4a8_kernel");
+    return;
+  }
+  if (M >= pair_min_rows()) {
+    const int bn = gemm_w8_pair_tile_width((static_cast<int64_t>(M) + 2 * kTileM - 1) / (2 * kTileM), N);
+    if (bn > 0) {
+      snprintf(name, cap, "gemm_w8a8_pair_kernel<%d>", bn);
+      return;
+    }
+  }
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  snprintf(name, cap, "gemm_w8a8_kernel<%d>", kTileN[choose_tile_n((static_cast<int64_t>(M) + kTileM - 1) / kTileM, N, sms)]);
+}
+
+static trdq_status launch_gemm_w8_mode(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, int mode,
+                                       const int32_t* const zp[2], cudaStream_t stream, int act = 0) {
+  const bool raw_i32 = mode == 1;
+  if (mode == 0 && static_cast<int64_t>(seg[0].M) + seg[1].M >= pair_min_rows()) {
     const trdq_status st = launch_gemm_w8_pair(w, g, seg, bias_bf16, stream, act);
     if (st != TRDQ_ERR_SHAPE) return st;
   }

@@ -58,6 +58,7 @@ struct alignas(64) Gemm2Params {
   const float* sw;
   const __nv_bfloat16* bias;
   int32_t N, K, tiles_n;
+  int32_t band;  // row tiles per band of the tile order; 0: column-block major over all row tiles
   uint32_t* status;
 };
 
@@ -65,9 +66,22 @@ struct TileCoord {
   int seg, m0, n0;
 };
 __device__ __forceinline__ TileCoord pair_tile_coord(const Gemm2Params& p, int tile, int bn) {
+  // Order of the tiles.  The clusters that run at the same time take consecutive tiles, so the order decides what they
+  // share in L2: within a band of `band` row tiles the tiles go column block by column block, i.e. a wave of clusters
+  // covers a band-high, many-columns-wide rectangle and re-reads few distinct panels of either operand.
   const int tiles_m = p.pair_tiles_m[0] + p.pair_tiles_m[1];
-  const int nt = tile / tiles_m;
-  int mt = tile - nt * tiles_m;
+  int nt, mt;
+  if (p.band <= 0) {
+    nt = tile / tiles_m;
+    mt = tile - nt * tiles_m;
+  } else {
+    const int per_band = p.band * p.tiles_n;
+    const int b = tile / per_band;
+    const int r = tile - b * per_band;
+    const int rows = min(p.band, tiles_m - b * p.band);
+    nt = r / rows;
+    mt = b * p.band + (r - nt * rows);
+  }
   TileCoord c;
   c.seg = mt >= p.pair_tiles_m[0] ? 1 : 0;
   if (c.seg) mt -= p.pair_tiles_m[0];
@@ -407,7 +421,130 @@ int max_clusters(int dev) {
   return known > 0 ? known : 0;
 }
 
+// Tile width: waves of resident clusters times the time of one tile.  The kernel is bound by operand delivery from L2,
+// so a tile costs what it loads, (256 + BN) panel rows of K bytes; wider tiles load less per multiply-add.  Checked
+// against a sweep of all three widths over the layer shapes at M = 4096 ... 32768: the model picks the fastest width or
+// one within 2 % of it (the earlier model, waves x (BN + 24), left 4 - 15 % on the table at M >= 16384).
+// Returns the index into kTileN (and the resident clusters of that width), or -1 if the kernel cannot run here.
+int pair_tile_choice(int64_t tiles_m, int N, int dev, int* clusters_out) {
+  int best = -1;
+  double best_cost = 1e300;
+  int clusters_of[kNumTileN];
+  for (int i = 0; i < kNumTileN; ++i) {
+    const int bn = kTileN[i];
+    clusters_of[i] = bn == 128 ? max_clusters<128>(dev) : bn == 192 ? max_clusters<192>(dev) : max_clusters<256>(dev);
+    if (clusters_of[i] <= 0) continue;
+    const int64_t tiles = tiles_m * ((N + bn - 1) / bn);
+    const int64_t waves = (tiles + clusters_of[i] - 1) / clusters_of[i];
+    const double cost = static_cast<double>(waves) * (256.0 + bn);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = i;
+    }
+  }
+  if (best >= 0 && clusters_out) *clusters_out = clusters_of[best];
+  return best;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Measurement aid: the tensor pipe by itself.  Every CTA pair issues `mmas` tcgen05.mma (256 x 256 x 32, int8) on
+// operands that already sit in shared memory, so there is no load and no epilogue: the rate this kernel reaches is the
+// ceiling any GEMM built on the instruction can approach on the device at its current clocks.
+// ---------------------------------------------------------------------------------------------
+constexpr int kCeilingThreads = 128;
+constexpr int kCeilingSmemBytes = 1024 + 2 * kTileM * kTileKBytes + 64;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kCeilingThreads, 1) mma_ceiling_kernel(int mmas, uint32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kTileM * kTileKBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
+  const uint32_t bar_done = smem_u32(bars);
+  const int warp = threadIdx.x >> 5;
+  const bool leader = cluster_ctarank() == 0;
+  // operands: 128 rows of A and this CTA's 128 rows of B, all ones (the layout does not matter for constant data)
+  for (int i = threadIdx.x; i < 2 * kTileM * kTileKBytes / 16; i += blockDim.x)
+    reinterpret_cast<uint4*>(smem)[i] = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+  if (threadIdx.x == 0) {
+    mbar_init(bar_done, 1);
+    fence_mbar_init();
+  }
+  fence_proxy_async_smem();
+  if (warp == 2) {
+    tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  BoundedWaiter w(status, kStatusTimeoutMma);
+  if (warp == 1 && leader && elect_one()) {
+    constexpr uint32_t idesc = umma_idesc_s8_pair(256);
+    const uint64_t a_desc = umma_desc_k_sw128(smem_base);
+    const uint64_t b_desc = umma_desc_k_sw128(smem_base + kTileM * kTileKBytes);
+    for (int i = 0; i < mmas; ++i) {
+      const int k = i & 3;
+      umma_i8_pair(tmem_base + ((i >> 2) & 1) * kAccStride, a_desc + 2 * k, b_desc + 2 * k, idesc, i >= 8 ? 1u : 0u);
+    }
+    umma_commit_pair(bar_done);
+  }
+  if (warp == 0) {
+    w.wait(bar_done, 0);  // arrives in both CTAs once every MMA has completed
+    w.settle();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 }  // namespace
+
+int gemm_w8_pair_tile_width(int64_t tiles_m, int N) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  const int i = pair_tile_choice(tiles_m, N, dev, nullptr);
+  return i < 0 ? 0 : kTileN[i];
+}
+
+trdq_status launch_mma_ceiling(int32_t mmas_per_cluster, int32_t* clusters_out, cudaStream_t stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRDQ_ERR_CUDA;
+  static PerDevice<int> cached;
+  int clusters = cached.get(dev);
+  if (clusters == 0) {
+    if (cudaFuncSetAttribute(mma_ceiling_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCeilingSmemBytes) != cudaSuccess) return TRDQ_ERR_CUDA;
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3(2);
+    q.blockDim = dim3(kCeilingThreads);
+    q.dynamicSmemBytes = kCeilingSmemBytes;
+    // one CTA per SM, as in the GEMM (a CTA holds all 512 tensor-memory columns): never more clusters than SM pairs
+    int sms = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, mma_ceiling_kernel, &q) != cudaSuccess || clusters <= 0 ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return TRDQ_ERR_CUDA;
+    }
+    if (clusters > sms / 2) clusters = sms / 2;
+    cached.set(dev, clusters);
+  }
+  uint32_t* status = device_status_word();
+  if (!status) return TRDQ_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * clusters);
+  cfg.blockDim = dim3(kCeilingThreads);
+  cfg.dynamicSmemBytes = kCeilingSmemBytes;
+  cfg.stream = stream;
+  if (cudaLaunchKernelEx(&cfg, mma_ceiling_kernel, static_cast<int>(mmas_per_cluster), status) != cudaSuccess) return TRDQ_ERR_CUDA;
+  if (clusters_out) *clusters_out = clusters;
+  return TRDQ_OK;
+}
 
 // Returns TRDQ_ERR_SHAPE when the pair kernel does not apply (caller falls back to the single-CTA kernel).
 trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16, cudaStream_t stream,
@@ -423,25 +560,8 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
     tiles_m += p.pair_tiles_m[s];
   }
   if (tiles_m == 0) return TRDQ_OK;
-  // Tile width: waves of resident clusters times the time of one tile.  The kernel is bound by operand delivery from L2,
-  // so a tile costs what it loads, (256 + BN) panel rows of K bytes; wider tiles load less per multiply-add.  Checked
-  // against a sweep of all three widths over the layer shapes at M = 4096 ... 32768: the model picks the fastest width or
-  // one within 2 % of it (the earlier model, waves x (BN + 24), left 4 - 15 % on the table at M >= 16384).
-  int best = -1;
-  double best_cost = 1e300;
-  int clusters_of[kNumTileN];
-  for (int i = 0; i < kNumTileN; ++i) {
-    const int bn = kTileN[i];
-    clusters_of[i] = bn == 128 ? max_clusters<128>(dev) : bn == 192 ? max_clusters<192>(dev) : max_clusters<256>(dev);
-    if (clusters_of[i] <= 0) continue;
-    const int64_t tiles = tiles_m * ((w->N + bn - 1) / bn);
-    const int64_t waves = (tiles + clusters_of[i] - 1) / clusters_of[i];
-    const double cost = static_cast<double>(waves) * (256.0 + bn);
-    if (cost < best_cost) {
-      best_cost = cost;
-      best = i;
-    }
-  }
+  int resident = 0;
+  const int best = pair_tile_choice(tiles_m, w->N, dev, &resident);
   if (best < 0) return TRDQ_ERR_SHAPE;
   const int bn = kTileN[best];
   for (int s = 0; s < 2; ++s) {
@@ -462,10 +582,13 @@ trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment 
   p.N = w->N;
   p.K = w->K;
   p.tiles_n = (w->N + bn - 1) / bn;
+  // Bands of four row tiles from 32 row tiles on (measured at M = 32768: +5 % on the K = 1152 layers, +22 % on
+  // 4608 -> 1152, any band height from 2 to 8 alike; at M = 4096 the plain column-block-major order is 1 % ahead).
+  p.band = tiles_m >= 32 ? 4 : 0;
   p.status = device_status_word();
   if (!p.status) return TRDQ_ERR_CUDA;
   const int64_t total = tiles_m * p.tiles_n;
-  const int clusters = static_cast<int>(total < clusters_of[best] ? total : clusters_of[best]);
+  const int clusters = static_cast<int>(total < resident ? total : resident);
   cudaError_t e;
   if (act)
     e = bn == 128 ? launch_pair<128, true>(p, clusters, stream) : bn == 192 ? launch_pair<192, true>(p, clusters, stream) : launch_pair<256, true>(p, clusters, stream);

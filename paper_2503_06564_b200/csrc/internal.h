@@ -120,6 +120,12 @@ trdq_status launch_gemm_w8_splitk(const trdq_weights* w, int g, const GemmSegmen
                                   int32_t* workspace, cudaStream_t stream);
 trdq_status launch_gemm_w8_splitk_static(const trdq_weights* w, int g, const GemmSegment& seg, const void* bias_bf16, int splits,
                                          cudaStream_t stream);
+// which kernel a call would run (for reports; the launchers use the same functions)
+void describe_rotate_quantize_kernel(int32_t M, int32_t K, char* name, size_t cap);
+void describe_gemm_kernel(int32_t M, int32_t K, int32_t N, int32_t wbits, char* name, size_t cap);
+int gemm_w8_pair_tile_width(int64_t pair_tiles_m, int N);  // 0: the pair kernel cannot run on this device
+// measurement aid: `mmas_per_cluster` back-to-back 256 x 256 x 32 int8 MMAs per CTA pair on resident operands
+trdq_status launch_mma_ceiling(int32_t mmas_per_cluster, int32_t* clusters_out, cudaStream_t stream);
 // gemm_i8_2cta.cu: CTA-pair kernel; TRDQ_ERR_SHAPE means "not applicable here, use the single-CTA kernel"
 trdq_status launch_gemm_w8_pair(const trdq_weights* w, int g, const GemmSegment seg[2], const void* bias_bf16,
                                 cudaStream_t stream, int act = 0);

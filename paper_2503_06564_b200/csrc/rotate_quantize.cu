@@ -13,6 +13,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdio>
 
 #include "internal.h"
 #include "lane_group.cuh"
@@ -687,6 +688,16 @@ cudaError_t launch_rotate2_quantize(const void* x_bf16, int64_t ldx, int32_t M, 
     rotate2_quantize_kernel<1><<<grid, threads, smem, stream>>>(static_cast<const __nv_bfloat16*>(x_bf16), ldx, M, K, vec1, perm, vec2,
                                                                 static_cast<int8_t*>(codes), static_cast<uint8_t*>(codes), scales, rows);
   return cudaGetLastError();
+}
+
+// Name of the kernel trdq_rotate_quantize runs for M rows of K channels (single rotation, symmetric codes).
+void describe_rotate_quantize_kernel(int32_t M, int32_t K, char* name, size_t cap) {
+  if (rotate_quantize_prefers_team(M, K))
+    snprintf(name, cap, "rotate_quantize_team_kernel");
+  else if (K / TRDQ_BLOCK <= 80 && static_cast<size_t>(K) * sizeof(float) <= 40 * 1024)
+    snprintf(name, cap, "rotate_quantize_rows_kernel");
+  else
+    snprintf(name, cap, "rotate_quantize_kernel");
 }
 
 cudaError_t launch_rotate_quantize(const void* x_bf16, int64_t ldx, int32_t M, int32_t K, const float* vec, int mode,

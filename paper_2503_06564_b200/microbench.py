@@ -4,6 +4,7 @@
     python -m paper_2503_06564_b200.microbench gemm --M 16384 --K 1152 --N 4608
     python -m paper_2503_06564_b200.microbench rqd  --M 16384 --K 1152      (dense block rotation, Eq. 6-8)
     python -m paper_2503_06564_b200.microbench nrq  --M 16384 --K 1152      (LayerNorm + modulation folded in front)
+    python -m paper_2503_06564_b200.microbench ceiling --mmas 65536         (tensor pipe alone: back-to-back MMAs on resident operands)
 
 Also the small, self-ending command to put under a profiler (few launches, a few hundred MB).
 Buffers are rotated through `--sets` distinct copies so that consecutive launches do not find
@@ -17,11 +18,30 @@ import json
 import numpy as np
 
 
+def mma_ceiling(mmas: int = 65536, iters: int = 10):
+    """Rate of the tensor pipe alone (TOPS): the best and the median of `iters` launches of the library's MMA-only kernel
+    (the rate scales with the SM clock the device runs at)."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    ops = trdq.trdq_measure_mma_ceiling(mmas)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    ev[0].record()
+    for i in range(iters):
+        trdq.trdq_measure_mma_ceiling(mmas)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(iters))
+    assert trdq.trdq_device_status() == 0
+    return {"kernel": "mma_ceiling_kernel", "mmas_per_cluster": mmas, "ops_per_launch": ops, "ms_median": ms[len(ms) // 2], "ms_min": ms[0],
+            "rate_median": ops / (ms[len(ms) // 2] * 1e-3) / 1e12, "rate_best": ops / (ms[0] * 1e-3) / 1e12, "unit": "TOPS"}
+
+
 def main():
     import torch
     from paper_2503_06564_b200 import build, trdq
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["rq", "rqd", "nrq", "gemm"])
+    ap.add_argument("kernel", choices=["rq", "rqd", "nrq", "gemm", "ceiling"])
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--K", type=int, default=1152)
     ap.add_argument("--N", type=int, default=4608)
@@ -29,11 +49,15 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--mmas", type=int, default=65536, help="ceiling: MMAs (256 x 256 x 32, int8) per CTA pair and launch")
     ap.add_argument("--full-transform", action="store_true", help="rq: rotation, zigzag permutation, second rotation (Eq. 9)")
     ap.add_argument("--splitk", action="store_true", help="gemm: use trdq_linear_splitk with a preallocated workspace")
     ap.add_argument("--no-graph", action="store_true", help="time individual launches issued from Python (profiler runs)")
     args = ap.parse_args()
     build.build()
+    if args.kernel == "ceiling":
+        print(json.dumps(mma_ceiling(args.mmas, args.iters)))
+        return
     torch.manual_seed(0)
     M, K, N = args.M, args.K, args.N
     rng = np.random.default_rng(0)

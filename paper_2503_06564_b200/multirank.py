@@ -6,7 +6,11 @@ on a time (max over ranks) and for barriers.
 """
 from __future__ import annotations
 
-from typing import Tuple
+import os
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence, Tuple
 
 
 def row_shard(M: int, rank: int, world: int, align: int = 1) -> Tuple[int, int]:
@@ -36,3 +40,48 @@ def max_over_ranks(value: float, device=None) -> float:
 def aggregate_rate(units_per_rank: float, world: int, ms: float) -> float:
     """Whole-job rate: every rank processed `units_per_rank` in `ms` (already the max over ranks)."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+def free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def rank_environment(rank: int, world: int, port: int, base: Optional[dict] = None) -> dict:
+    """Environment of one rank of a single-node job: what a torchrun launch would have set."""
+    env = dict(os.environ if base is None else base)
+    env.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), LOCAL_WORLD_SIZE=str(world),
+               MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    return env
+
+
+def spawn_ranks(world: int, argv: Sequence[str], timeout: Optional[float] = None) -> Tuple[int, str]:
+    """Runs `argv` (a command line) as `world` processes of one node, one per rank, each with the
+    rendezvous variables of `rank_environment`.  Rank 0's standard output is captured and returned;
+    the other ranks' output goes to this process's stderr.  Returns (worst exit code, rank 0's stdout).
+    A rank that fails or overruns `timeout` seconds ends the others (by PID)."""
+    if world < 1:
+        raise ValueError("world size must be positive")
+    port = free_port()
+    procs: List[subprocess.Popen] = []
+    for rank in range(world):
+        procs.append(subprocess.Popen(list(argv), env=rank_environment(rank, world, port),
+                                      stdout=subprocess.PIPE if rank == 0 else sys.stderr, text=rank == 0))
+    worst, out0 = 0, ""
+    try:
+        out0, _ = procs[0].communicate(timeout=timeout)
+        worst = procs[0].returncode
+        for p in procs[1:]:
+            rc = p.wait(timeout=timeout)
+            worst = worst or rc
+    except subprocess.TimeoutExpired:
+        worst = 124
+    finally:
+        for p in procs:
+            if p.poll() is None:
+                p.kill()
+                p.wait()
+    return worst, out0

@@ -30,7 +30,8 @@ EXPORTS = (
     "trdq_run_layers", "trdq_linear_splitk_workspace", "trdq_linear_splitk", "trdq_linear_splitk_static",
     "trdq_rotation_create_full", "trdq_zigzag_permutation", "trdq_rotate_quantize_asym", "trdq_linear_asym",
     "trdq_selftest_wait_expiry", "trdq_rotation_create_dense", "trdq_rotate_dense_workspace", "trdq_rotate_dense_quantize",
-    "trdq_greedy_rotation_block", "trdq_linear_act", "trdq_norm_rotate_quantize",
+    "trdq_greedy_rotation_block", "trdq_linear_act", "trdq_norm_rotate_quantize", "trdq_kernel_choice",
+    "trdq_measure_mma_ceiling",
 )
 
 
@@ -80,6 +81,8 @@ def lib() -> C.CDLL:
         l.trdq_linear.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, vp]
         l.trdq_norm_rotate_quantize.argtypes = [vp, i32, vp, i64, i32, vp, vp, i32, C.c_float, vp, vp, vp]
         l.trdq_linear_act.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i32, vp]
+        l.trdq_kernel_choice.argtypes = [i32, i32, i32, i32, i32, C.c_char_p, i32]
+        l.trdq_measure_mma_ceiling.argtypes = [i32, C.POINTER(i32), vp]
         l.trdq_linear_cfg.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32), vp, C.POINTER(vp),
                                       C.POINTER(i64), vp]
         l.trdq_gemm_i32.argtypes = [vp, i32, vp, i32, vp, i64, vp]
@@ -461,6 +464,20 @@ def trdq_run_layers(layers: LayerList, t: int, first: int = 0, count: Optional[i
     arr = layers.array()
     ptr = C.cast(C.byref(arr, first * C.sizeof(LayerOp)), C.POINTER(LayerOp))
     _check(lib().trdq_run_layers(ptr, int(n), int(t), _stream()), "trdq_run_layers")
+
+
+def trdq_kernel_choice(stage: int, M: int, K: int, N: int = 0, wbits: int = 8) -> str:
+    """Name of the kernel trdq_rotate_quantize (stage 0) or trdq_linear (stage 1) runs for this shape on the current device."""
+    buf = C.create_string_buffer(96)
+    _check(lib().trdq_kernel_choice(int(stage), int(M), int(K), int(N), int(wbits), buf, 96), "trdq_kernel_choice")
+    return buf.value.decode()
+
+
+def trdq_measure_mma_ceiling(mmas_per_cluster: int) -> int:
+    """Launches the tensor-pipe-only kernel on the current stream; returns the integer operations the launch performs."""
+    clusters = C.c_int32(0)
+    _check(lib().trdq_measure_mma_ceiling(int(mmas_per_cluster), C.byref(clusters), _stream()), "trdq_measure_mma_ceiling")
+    return clusters.value * int(mmas_per_cluster) * 2 * 256 * 256 * 32
 
 
 def trdq_selftest_wait_expiry() -> None:

@@ -71,3 +71,30 @@ def test_two_ranks_shard_rows_without_collective(tmp_path):
 
 def test_max_over_ranks_without_process_group():
     assert multirank.max_over_ranks(3.5) == 3.5
+
+
+def test_spawn_ranks_gives_every_rank_its_environment(tmp_path):
+    """The launcher bench.py uses when it is asked for N GPUs outside torchrun: N processes with RANK / WORLD_SIZE /
+    MASTER_* set, which can form a process group (gloo here) and agree on a maximum; rank 0's output is returned."""
+    import sys
+    script = tmp_path / "rank.py"
+    script.write_text(
+        "import os, sys\n"
+        f"sys.path.insert(0, {repr(os.path.dirname(os.path.dirname(os.path.abspath(__file__))))})\n"
+        "import torch.distributed as dist\n"
+        "from paper_2503_06564_b200 import multirank\n"
+        "rank, world = int(os.environ['RANK']), int(os.environ['WORLD_SIZE'])\n"
+        "assert os.environ['MASTER_ADDR'] == '127.0.0.1' and int(os.environ['LOCAL_RANK']) == rank\n"
+        "dist.init_process_group('gloo', rank=rank, world_size=world)\n"
+        "t = multirank.max_over_ranks(1.0 + rank)\n"
+        "dist.barrier()\n"
+        "dist.destroy_process_group()\n"
+        "if rank == 0: print('world', world, 'max', t)\n")
+    rc, out = multirank.spawn_ranks(2, [sys.executable, str(script)], timeout=120)
+    assert rc == 0 and out.strip() == "world 2 max 2.0"
+    bad = tmp_path / "bad.py"
+    bad.write_text("import os, sys\nsys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
+    rc, _ = multirank.spawn_ranks(2, [sys.executable, str(bad)], timeout=60)
+    assert rc == 3
+    with pytest.raises(ValueError):
+        multirank.spawn_ranks(0, [sys.executable, str(bad)])
