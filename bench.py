@@ -29,8 +29,8 @@ METRIC = "rotated_w8a8_linear_tops"
 UNIT = "TOPS"
 # DRAM traffic per unit of algorithmic work, from the Nsight Compute captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch); None once a kernel has changed since its capture.
-GEMM_PAIR_DRAM_BYTES_PER_OP = 123.3e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
-RQ_TEAM_DRAM_BYTES_PER_ALG_BYTE = None              # rotate_quantize_team_kernel: set from its capture under profiles/
+GEMM_PAIR_DRAM_BYTES_PER_OP = 116.3e6 / 174.0e9     # gemm_w8a8_pair_kernel, M = 16384, K = 1152, N = 4608
+RQ_TEAM_DRAM_BYTES_PER_ALG_BYTE = 659.6 / 793.3     # rotate_quantize_team_kernel, M = 32768: three K = 1152 launches and one K = 4608
 INT8_OVER_BF16 = 2.0          # nominal dense INT8 : bf16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -556,10 +556,14 @@ def run_ours(args, wl: WL.Workload):
     time.sleep(0.0 if args.quick else 1.0)
     ms_rq_b, sec_rq_b = rq_pass.ms(min_seconds=0.25)
     assert trdq.trdq_device_status() == 0, "a bounded device-side wait expired during the benchmark"
-    roof_gemm, roof_rq, per_layer = roofline_entries(wl, peaks, ops, ms_gemm, sec_gemm, ms_rq, sec_rq, dense)
-    burst_gemm, burst_rq, _ = roofline_entries(wl, peaks, ops, ms_gemm_b, sec_gemm_b, ms_rq_b, sec_rq_b, dense)
+    # GEMM: the two-second pass against the sustained tensor peak is the headline, the brief pass against the burst peak
+    # beside it.  Rotate + quantize: the one measured copy rate is a best-of-ten of millisecond copies, i.e. a burst
+    # figure, so the brief pass is the like-for-like headline and the two-second pass is reported beside it.
+    roof_gemm, rq_long, per_layer = roofline_entries(wl, peaks, ops, ms_gemm, sec_gemm, ms_rq, sec_rq, dense)
+    burst_gemm, roof_rq, _ = roofline_entries(wl, peaks, ops, ms_gemm_b, sec_gemm_b, ms_rq_b, sec_rq_b, dense)
     roof_gemm["brief"] = {k: burst_gemm[k] for k in ("achieved", "peak", "frac", "frac_nominal", "seconds_timed", "peak_source")}
-    roof_rq["brief"] = {k: burst_rq[k] for k in ("achieved", "frac", "frac_nominal", "seconds_timed")}
+    roof_rq["sustained"] = {k: rq_long[k] for k in ("achieved", "frac", "frac_nominal", "seconds_timed")}
+    roof_rq["peak_source"] += " (best of ten 4 GB copies: a burst figure, compared with the brief pass)"
     ceiling = None
     if rank == 0 and wl.wbits == 8:
         c = microbench.mma_ceiling(65536, 5)
@@ -627,7 +631,8 @@ def run_ours(args, wl: WL.Workload):
         "us_per_dit_step": ms_per_step * 1e3,
         "rotate_quantize_gbs": roof_rq["achieved"],
         "gemm_tops": roof_gemm["achieved"],
-        "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm},
+        "kernel_ms_per_step": {"rotate_quantize": ms_rq, "gemm_epilogue": ms_gemm, "what": "two-second passes of one kernel kind",
+                               "brief": {"rotate_quantize": ms_rq_b, "gemm_epilogue": ms_gemm_b}},
         "sustained": {"ms_per_step": ms_sustained, "steps": reps_long, "tops": ops / (ms_sustained * 1e-3) / 1e12,
                       "clocks": clocks_sustained, "what": "the same step loop run for at least two seconds, after the per-kernel passes"},
         "roofline": roof_gemm,
