@@ -367,6 +367,9 @@ trdq_status trdq_prepare_weights(const trdq_rotation* rot, const void* W_bf16, i
         return TRDQ_ERR_CUDA;
       }
     }
+    // The kernels below end the group's preparation and MUST stay ordinary launches (full stream dependency, no early
+    // trigger of dependents): the GEMM kernels request weight tiles before their dependent-launch wait, which orders
+    // them only against the kernel directly before them, so the codes have to be complete before that kernel starts.
     if (wbits == 8) {
       if (cudaMalloc(&gw.colsum, static_cast<size_t>(N) * sizeof(int32_t)) != cudaSuccess) {
         cudaGetLastError();

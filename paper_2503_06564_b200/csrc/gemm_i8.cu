@@ -147,6 +147,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_w8a8_kernel(const __grid_con
   griddep_launch_dependents();
   // The weights are constants of the prepared object: the weight tiles of the first tile's first stages are requested
   // before waiting for the kernel before (which produced the activation codes), so their latency overlaps its tail.
+  // RULE this relies on: griddepcontrol.wait orders this kernel only against its immediate predecessor in the stream, so
+  // the weight codes must be complete before that predecessor can start.  trdq_prepare_weights guarantees it: the last
+  // kernel it enqueues per group (column sums / 4-bit multipliers, or a stream synchronisation for dense rotations) is
+  // launched the ordinary way, i.e. with a full dependency on the kernels that wrote the codes, and never triggers its
+  // dependents early.
   int prefetched = 0;
   if (static_cast<int>(blockIdx.x) < total_tiles) {
     const TileCoord tc0 = tile_coord(p, blockIdx.x, BN);

@@ -205,6 +205,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_w8
   griddep_launch_dependents();
   // The weights are constants of the prepared object, so the weight halves of the first tile's first stages are requested
   // before waiting for the kernel before (which produced the activation codes): their latency overlaps its tail.
+  // RULE this relies on: griddepcontrol.wait orders this kernel only against its immediate predecessor in the stream, so
+  // the weight codes must be complete before that predecessor can start.  trdq_prepare_weights guarantees it: the last
+  // kernel it enqueues per group (column sums / 4-bit multipliers, or a stream synchronisation for dense rotations) is
+  // launched the ordinary way, i.e. with a full dependency on the kernels that wrote the codes, and never triggers its
+  // dependents early.
   const int prefetched = cluster_id < total_tiles ? min(C::kStages, num_kb) : 0;
   if (threadIdx.x == 0) {
     const uint32_t leader_full0 = map_to_cta(bar_full, 0);

@@ -455,3 +455,41 @@ def test_every_linear_entry_point_validates_on_the_host():
     assert lib.trdq_linear_splitk_static(h, 0, c, sc, M, bias_odd.data_ptr() + 2, yp, N, st) == 0
     assert torch.equal(y, expected)
     assert trdq.trdq_device_status() == 0
+
+
+def test_prepare_then_use_on_one_stream_without_synchronisation():
+    """Weight preparation, rotate + quantize and the linear enqueued back to back on one stream, nothing synchronised in
+    between, several fresh weight sets in a row: the GEMM requests weight tiles before its dependent-launch wait, which
+    is only correct if the preparation's last kernel fully orders the code-writing kernels before anything that follows."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(77)
+    M, K = 2304, 1152                                   # enough rows for the CTA-pair kernel
+    x_bits = _acts(M, K, 78)
+    xd = to_dev_bf16(x_bits)
+    rows = np.arange(0, M, 53, dtype=np.int64)
+    signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
+    rot = trdq.Rotation(K, [0, 1000], signs)
+    act, wv = O.fused_vectors(signs[0], None)
+    q_ref, sx_ref = O.rotate_quantize(x_bits, act)
+    cases = []
+    for i, (N, wbits) in enumerate([(1152, 8), (256, 8), (3456, 8), (640, 4), (1152, 8), (128, 8)]):
+        w_bits = WL.to_bf16_bits(rng.standard_normal((N, K)) * 0.03)
+        bias_bits = WL.to_bf16_bits(rng.standard_normal(N) * 0.01)
+        cases.append((N, wbits, w_bits, bias_bits, to_dev_bf16(w_bits), to_dev_bf16(bias_bits)))
+    torch.cuda.synchronize()
+    outs = []
+    for N, wbits, w_bits, bias_bits, wd, bd in cases:    # no synchronisation from here to the end of the loop
+        wts = trdq.trdq_prepare_weights(rot, wd, wbits)
+        codes, scales = trdq.trdq_rotate_quantize(rot, 0, xd)
+        outs.append((wts, trdq.trdq_linear(wts, 0, codes, scales, bd)))
+    torch.cuda.synchronize()
+    for (N, wbits, w_bits, bias_bits, wd, bd), (wts, y) in zip(cases, outs):
+        if wbits == 8:
+            qw, sw = O.prepare_w8(w_bits, wv)
+            y_ref = O.linear_w8_rows(q_ref, sx_ref, qw, sw, bias_bits, rows)
+        else:
+            pk, sw4 = O.prepare_w4(w_bits, wv)
+            y_ref = O.linear_w4_rows(q_ref, sx_ref, pk, sw4, bias_bits, rows)
+        check_output(bf16_to_f32_np(y)[rows], y_ref)
+    assert trdq.trdq_device_status() == 0
