@@ -28,7 +28,9 @@
  *     forms, trdq_run_layers, trdq_gemm_i32) allocate no memory; trdq_prepare_weights with a
  *     dense-block rotation is the one call that waits for its own work (it frees a scratch buffer).
  *   - The caller owns every tensor it passes.  The library owns only the opaque
- *     trdq_rotation / trdq_weights objects until their _destroy call.
+ *     trdq_rotation / trdq_weights objects until their _destroy call.  An object belongs to the
+ *     device that was current when it was created; calls that use it with another device
+ *     current return TRDQ_ERR_MISMATCH.  Entry points may be called from several host threads.
  *   - Errors are reported by return code only; the library never aborts, traps or
  *     prints.  Argument errors are found on the host before anything is launched.
  *     NaN/Inf in X or W give unspecified codes (not checked).
@@ -58,7 +60,8 @@ typedef enum trdq_status {
   TRDQ_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (no device, launch error, ...) */
   TRDQ_ERR_NOMEM = 8,     /* host or device allocation failed */
   TRDQ_ERR_TIMEOUT = 9,   /* a bounded device-side wait expired (see trdq_device_status) */
-  TRDQ_ERR_MISMATCH = 10, /* objects passed together were built for different K / groups, or the rotation's kind does not fit the call */
+  TRDQ_ERR_MISMATCH = 10, /* objects passed together were built for different K / groups, the rotation's kind does not fit the call,
+                             or the current device is not the one the object was created on */
   TRDQ_ERR_SCRATCH = 11   /* the problem needs more than the library's built-in scratch area (trdq_linear_splitk_static) */
 } trdq_status;
 
