@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "internal.h"
@@ -34,34 +35,81 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
+  static const EncodeTiledFn fn = [] {   // initialised once, also under concurrent first calls
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
   return fn;
+}
+
+// Encoded tensor maps are remembered by their full description: a caller that issues the same layer step after
+// step without a CUDA graph re-describes the same buffers every call (two maps per rotate + quantize, four to six per
+// GEMM), and an encode costs about a microsecond of host time.  Direct-mapped, 512 entries, one mutex; a map is a pure
+// function of its key, so a stale entry cannot exist: a freed and reused address with the same shape gives the same map.
+struct TmapKey {
+  const void* base;
+  uint64_t dims[3];
+  uint64_t strides[2];
+  uint32_t box[3];
+  uint32_t rank, dtype, swizzle;
+};
+struct TmapEntry {
+  bool valid = false;
+  TmapKey key;
+  CUtensorMap map;
+};
+static std::mutex g_tmap_mutex;
+static TmapEntry g_tmap_cache[512];
+
+static trdq_status encode_cached(CUtensorMap* out, CUtensorMapDataType dt, uint32_t rank, const void* base, const cuuint64_t* dims,
+                                 const cuuint64_t* strides, const cuuint32_t* box, CUtensorMapSwizzle sw) {
+  TmapKey key;
+  std::memset(&key, 0, sizeof key);
+  key.base = base;
+  key.rank = rank;
+  key.dtype = static_cast<uint32_t>(dt);
+  key.swizzle = static_cast<uint32_t>(sw);
+  for (uint32_t i = 0; i < rank; ++i) {
+    key.dims[i] = dims[i];
+    key.box[i] = box[i];
+    if (i + 1 < rank) key.strides[i] = strides[i];
+  }
+  uint64_t h = 1469598103934665603ull;
+  const unsigned char* kb = reinterpret_cast<const unsigned char*>(&key);
+  for (size_t i = 0; i < sizeof key; ++i) h = (h ^ kb[i]) * 1099511628211ull;
+  TmapEntry& slot = g_tmap_cache[h & 511u];
+  {
+    std::lock_guard<std::mutex> lock(g_tmap_mutex);
+    if (slot.valid && std::memcmp(&slot.key, &key, sizeof key) == 0) {
+      *out = slot.map;
+      return TRDQ_OK;
+    }
+  }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return TRDQ_ERR_CUDA;
+  const cuuint32_t elem_strides[3] = {1, 1, 1};
+  const CUresult r = fn(out, dt, rank, const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return TRDQ_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_tmap_mutex);
+  slot.key = key;
+  slot.map = *out;
+  slot.valid = true;
+  return TRDQ_OK;
 }
 
 trdq_status encode_tmap_u8_sw128(CUtensorMap* out, const void* base, uint64_t row_bytes, uint64_t rows,
                                  uint64_t row_stride_bytes, uint32_t box_bytes, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return TRDQ_ERR_CUDA;
   const cuuint64_t dims[2] = {row_bytes, rows};
   const cuuint64_t strides[1] = {row_stride_bytes};
   const cuuint32_t box[2] = {box_bytes, box_rows};
-  const cuuint32_t elem_strides[2] = {1, 1};
-  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return encode_cached(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint64_t cols, uint64_t rows,
                            uint64_t row_stride_bytes, uint32_t box_cols, uint32_t box_rows, uint32_t swizzle_bytes) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return TRDQ_ERR_CUDA;
   const CUtensorMapDataType dt = elem_bytes == 1   ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                  : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16
                                                    : CU_TENSOR_MAP_DATA_TYPE_UINT32;
@@ -72,24 +120,16 @@ trdq_status encode_tmap_2d(CUtensorMap* out, const void* base, uint32_t elem_byt
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {row_stride_bytes};
   const cuuint32_t box[2] = {box_cols, box_rows};
-  const cuuint32_t elem_strides[2] = {1, 1};
-  const CUresult r = fn(out, dt, 2, const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return encode_cached(out, dt, 2, base, dims, strides, box, sw);
 }
 
 trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_bytes, uint32_t box_cols, uint64_t rows,
                               uint64_t row_stride_bytes, uint32_t boxes, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return TRDQ_ERR_CUDA;
   const CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16;
   const cuuint64_t dims[3] = {box_cols, rows, boxes};
   const cuuint64_t strides[2] = {row_stride_bytes, static_cast<cuuint64_t>(box_cols) * elem_bytes};
   const cuuint32_t box[3] = {box_cols, box_rows, boxes};
-  const cuuint32_t elem_strides[3] = {1, 1, 1};
-  const CUresult r = fn(out, dt, 3, const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return encode_cached(out, dt, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

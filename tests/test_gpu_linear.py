@@ -261,7 +261,7 @@ def test_small_shapes_through_the_cta_pair_kernel():
     env = dict(os.environ, TRDQ_PAIR_MIN_M="1")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     res = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-m", "gpu", "-x", "-q", "-k",
-                          "not w4a8 and not through_the_cta_pair", "--timeout", "300"], cwd=root, env=env,
+                          "not w4a8 and not through_the_cta_pair"], cwd=root, env=env,
                          capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
 
@@ -493,3 +493,33 @@ def test_prepare_then_use_on_one_stream_without_synchronisation():
             y_ref = O.linear_w4_rows(q_ref, sx_ref, pk, sw4, bias_bits, rows)
         check_output(bf16_to_f32_np(y)[rows], y_ref)
     assert trdq.trdq_device_status() == 0
+
+
+def test_kernel_choice_and_tensor_pipe_ceiling():
+    """The two reporting aids: the library names the kernel a shape gets (the same functions the launchers use), and
+    the MMA-only kernel runs to completion and reports the operations it performed."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    assert trdq.trdq_kernel_choice(0, 256, 1024) == "rotate_quantize_rows_kernel"
+    assert trdq.trdq_kernel_choice(0, 32768, 1152) == "rotate_quantize_team_kernel"
+    assert trdq.trdq_kernel_choice(0, 8, 17408) == "rotate_quantize_kernel"
+    assert trdq.trdq_kernel_choice(1, 32768, 1152, 4608, 8).startswith("gemm_w8a8_pair_kernel<")
+    import os
+    small_is_pair = int(os.environ.get("TRDQ_PAIR_MIN_M", "2048")) <= 960      # the child run of this file lowers the threshold
+    assert trdq.trdq_kernel_choice(1, 960, 4096, 1152, 8).startswith("gemm_w8a8_pair_kernel<" if small_is_pair else "gemm_w8a8_kernel<")
+    assert trdq.trdq_kernel_choice(1, 16384, 1152, 4608, 4) == "gemm_w4a8_kernel"
+    with pytest.raises(trdq.TrdqError) as e:
+        trdq.trdq_kernel_choice(1, 128, 1152, 1152, 6)
+    assert e.value.status == 6
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    trdq.trdq_measure_mma_ceiling(4096)
+    e0.record()
+    ops = trdq.trdq_measure_mma_ceiling(16384)
+    e1.record()
+    torch.cuda.synchronize()
+    assert trdq.trdq_device_status() == 0
+    tops = ops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    per_cluster = 16384 * 2 * 256 * 256 * 32
+    assert ops % per_cluster == 0 and 1 <= ops // per_cluster <= sms // 2
+    assert 1000.0 < tops < 6000.0, tops           # the tensor pipe alone: a few PTOPS on this part

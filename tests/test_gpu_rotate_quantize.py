@@ -38,10 +38,16 @@ def _x(M, K, seed, outliers=True):
     (100, 640, 2, True),        # 5 blocks: 56 rows per tile, the last warp is partly idle, ragged last tile
     (9, 4736, 1, True),         # 37 blocks: too wide for one thread per block, lane-group kernel
     (600, 1152, 1, False),
-    (9500, 1152, 1, True),      # 297 tiles of 32 rows: still the lane-group kernel (fewer than six rounds of one tile per SM)
-    (28500, 1152, 1, True),     # enough rows for the one-thread-per-block TMA kernel: 891 tiles, ring wraps, ragged tail
-    (7200, 4608, 1, False),     # same kernel, 36 blocks, 8 rows per tile
-    (50000, 640, 2, True),      # same kernel, 5 blocks: 56 rows per tile, partly idle last warp
+    (9500, 1152, 1, True),      # team kernel, one-warp teams of 3 rows (27 of 32 lanes): 3167 tiles over 1776 teams, ragged tail
+    (28500, 1152, 1, True),     # same, five to six tiles per team: both ring stages wrap several times
+    (2100, 1152, 1, True),      # too few tiles for one-warp teams: two-warp teams of 7 rows (named barrier between the warps)
+    (7200, 4608, 1, False),     # 36 blocks: four-warp teams of 3 rows, three teams per CTA
+    (50000, 640, 2, True),      # 5 blocks: one-warp teams of 6 rows, eleven teams (shared memory bound)
+    (4000, 4096, 1, True),      # 32 blocks: one row per warp, ten teams
+    (5000, 2048, 1, False),     # 16 blocks: two rows per warp
+    (3000, 8192, 1, True),      # 64 blocks: two-warp teams of one row
+    (1500, 10240, 1, True),     # 80 blocks: three-warp teams of one row (80 of 96 lanes), three teams
+    (149, 1152, 1, True),       # just over one tile per SM with the widest team: team kernel, most teams idle
 ])
 def test_rotate_quantize_matches_oracle(M, K, G, smooth):
     from paper_2503_06564_b200 import trdq
@@ -87,6 +93,44 @@ def test_rotate_quantize_strided_rows_zero_rows_and_group_switch():
     assert torch.equal(a, b)
     # M == 0 is a no-op
     trdq.trdq_rotate_quantize(rot, 0, wide[:0, :K])
+
+
+def test_team_kernel_strided_rows_zero_rows_and_ties():
+    """The same special cases at row counts that go to the one-thread-per-block team kernel: a row stride wider than K,
+    all-zero tokens scattered through the tiles (scale 0, codes 0), and exact rounding ties (half to even)."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    K, M = 1152, 9001
+    assert trdq.trdq_kernel_choice(0, M, K) == "rotate_quantize_team_kernel"
+    rot, signs, sm, bounds = _rot(K, 1, 5, True)
+    x = _x(M, K, 10)
+    zero_rows = [0, 4, 5, 3000, M - 1]
+    x[zero_rows] = 0
+    wide = torch.zeros((M, K + 128), dtype=torch.bfloat16, device="cuda")
+    wide[:, :K] = to_dev_bf16(x)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, wide[:, :K])
+    act, _ = O.fused_vectors(signs[0], sm[0])
+    c_ref, s_ref = O.rotate_quantize(x, act)
+    assert np.array_equal(codes.cpu().numpy(), c_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+    assert not scales[zero_rows].any().item() and not codes[zero_rows].any().item()
+    # ties: the five exact rows of test_rounding_ties_on_device repeated 2000 times (K = 128: 32 rows per one-warp team)
+    K2, reps = 128, 2000
+    assert trdq.trdq_kernel_choice(0, 5 * reps, K2) == "rotate_quantize_team_kernel"
+    rot2 = trdq.Rotation(K2, [0, 1000], np.ones((1, K2), np.int8), np.full((1, K2), np.float32(2.0 ** 3.5), np.float32))
+    base = np.zeros((5, K2))
+    base[0, :4] = [201, 150, 99, 58]
+    base[1, :4] = [-201, -150, -99, -58]
+    base[2, :2] = [255, 253]
+    base[3, :4] = [131, 130, 126, 121]
+    base[4, :4] = [-131, -130, -126, -121]
+    xb = WL.to_bf16_bits(np.tile(base, (reps, 1)))
+    c2, s2 = trdq.trdq_rotate_quantize(rot2, 0, to_dev_bf16(xb))
+    c2 = c2.cpu().numpy().reshape(reps, 5, K2)
+    assert np.all(s2.cpu().numpy() == 4.0)
+    i = np.arange(K2) & 3
+    expect = np.stack([np.array(v)[i] for v in ([127, 23, 48, 2], [-127, -23, -48, -2], [127, 0, 127, 0], [127, 2, 4, -1], [-127, -2, -4, 1])])
+    assert np.array_equal(c2, np.broadcast_to(expect, c2.shape))
+    assert trdq.trdq_device_status() == 0
 
 
 def test_rounding_ties_on_device():

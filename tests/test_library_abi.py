@@ -90,6 +90,16 @@ def test_host_side_validation_needs_no_device(lib):
     assert lib.trdq_linear_splitk_static(None, 0, None, None, 0, None, None, 0, None) == 1
     assert lib.trdq_linear_splitk_workspace(None, 0, None, None) == 1
     assert lib.trdq_linear_asym(None, 0, None, None, None, 0, None, None, 0, None) == 1
+    # reporting aids: argument checks come before any device query
+    name = C.create_string_buffer(96)
+    assert lib.trdq_kernel_choice(0, 128, 1152, 0, 8, None, 96) == 1
+    assert lib.trdq_kernel_choice(0, 128, 1152, 0, 8, name, 8) == 2          # buffer too small for a kernel name
+    assert lib.trdq_kernel_choice(0, 0, 1152, 0, 8, name, 96) == 2
+    assert lib.trdq_kernel_choice(0, 128, 1000, 0, 8, name, 96) == 2         # K not a multiple of the block
+    assert lib.trdq_measure_mma_ceiling(1024, None, None) == 1
+    clusters = C.c_int32(0)
+    assert lib.trdq_measure_mma_ceiling(4, C.byref(clusters), None) == 2     # fewer than eight MMAs
+    assert lib.trdq_measure_mma_ceiling(1 << 23, C.byref(clusters), None) == 2
     assert lib.trdq_rotation_destroy(None) == 0 and lib.trdq_weights_destroy(None) == 0
     import torch
     if not torch.cuda.is_available():
