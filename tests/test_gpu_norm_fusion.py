@@ -31,7 +31,10 @@ def reference(x_bits, shift_bits, scale_bits, rps, eps, act_vec):
     return v, tol_v
 
 
-@pytest.mark.parametrize("M,K,rps,G", [(300, 1152, 64, 2), (37, 4608, 16, 1), (5, 128, 2, 1), (1024, 1152, 256, 1), (64, 8192, 64, 1)])
+@pytest.mark.parametrize("M,K,rps,G", [(300, 1152, 64, 2), (37, 4608, 16, 1), (5, 128, 2, 1), (1024, 1152, 256, 1), (64, 8192, 64, 1),
+                                       # thousands of rows: samples that are not a multiple of the row tile, a ragged last sample,
+                                       # 32- and 36-block rows, and samples of only four rows
+                                       (8192, 1152, 256, 2), (5000, 1152, 1000, 1), (3000, 4096, 64, 1), (2400, 4608, 100, 1), (4000, 1152, 4, 1)])
 def test_norm_fused_codes_match_oracle(M, K, rps, G):
     from paper_2503_06564_b200 import trdq
     rng = np.random.default_rng(200 + K + M)
@@ -84,6 +87,17 @@ def test_norm_fused_exact_rows_and_determinism():
     assert set(np.unique(h)) <= {np.float32(0.75), np.float32(-0.25)}
     c_ref, s_ref = O.quantize_rows(O.rotate_f32(h, a))
     assert np.array_equal(codes.cpu().numpy(), c_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+    # the same exact rows sixty times over, in samples of 70 rows (35 rows of each sign pattern pair do not align with any row tile)
+    reps = 60
+    xb_big = np.tile(x_bits, (reps, 1))
+    cb, sb = trdq.trdq_norm_rotate_quantize(rot, 0, to_dev_bf16(xb_big), to_dev_bf16(np.tile(shift_bits, (35, 1))),
+                                            to_dev_bf16(np.tile(scale_bits, (35, 1))), 70, 0.0)
+    assert np.array_equal(cb.cpu().numpy(), np.tile(c_ref, (reps, 1))) and np.array_equal(sb.cpu().numpy(), np.tile(s_ref, reps))
+    xr_big = to_dev_bf16(WL.to_bf16_bits(rng.standard_normal((M * reps, K)) * 3.0))
+    c1, s1 = trdq.trdq_norm_rotate_quantize(rot, 0, xr_big, None, None, 70, 1e-6)
+    for _ in range(3):
+        c2, s2 = trdq.trdq_norm_rotate_quantize(rot, 0, xr_big, None, None, 70, 1e-6)
+        assert torch.equal(c1, c2) and torch.equal(s1, s2)
     # determinism on ordinary data
     xr = to_dev_bf16(WL.to_bf16_bits(rng.standard_normal((M, K)) * 3.0))
     c1, s1 = trdq.trdq_norm_rotate_quantize(rot, 0, xr, None, None, M, 1e-6)
