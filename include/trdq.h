@@ -36,6 +36,10 @@
  *     NaN/Inf in X or W give unspecified codes (not checked).
  *   - There is no CPU fallback: without a CUDA device every call that needs one
  *     returns TRDQ_ERR_CUDA.
+ *   - Debug runs: with TRDQ_DEBUG=1 in the environment (read once per process) every online call waits
+ *     for its own work and returns TRDQ_ERR_CUDA / TRDQ_ERR_TIMEOUT itself if the device reported an
+ *     error or a bounded wait expired (the status word is read and cleared), so a problem is pinned to
+ *     the call that caused it.  Such a process must not capture those calls into a CUDA graph.
  */
 #ifndef TRDQ_H_
 #define TRDQ_H_

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -130,6 +131,23 @@ trdq_status encode_tmap_boxes(CUtensorMap* out, const void* base, uint32_t elem_
   const cuuint64_t strides[2] = {row_stride_bytes, static_cast<cuuint64_t>(box_cols) * elem_bytes};
   const cuuint32_t box[3] = {box_cols, box_rows, boxes};
   return encode_cached(out, dt, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// TRDQ_DEBUG=1 (read once per process): every online call waits for its own work and reports what the device did with it:
+// a CUDA error becomes TRDQ_ERR_CUDA at the call that caused it, an expired bounded wait TRDQ_ERR_TIMEOUT (the status word
+// is read and cleared).  The stand-in for a sanitizer run: the kernels clip every access by construction (TMA boxes, row and
+// column guards), so what a debug run adds is WHERE something went wrong.  Not usable while a stream is being captured.
+static bool debug_mode() {
+  static const bool on = [] {
+    const char* e = getenv("TRDQ_DEBUG");
+    return e && e[0] != '\0' && e[0] != '0';
+  }();
+  return on;
+}
+trdq_status finish(trdq_status st, void* stream) {
+  if (st != TRDQ_OK || !debug_mode()) return st;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess || cudaGetLastError() != cudaSuccess) return TRDQ_ERR_CUDA;
+  return trdq_device_status(nullptr);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -501,12 +519,12 @@ trdq_status trdq_rotate_quantize(const trdq_rotation* rot, int32_t t, const void
     const cudaError_t e2 = launch_rotate2_quantize(X_bf16, ldx, M, rot->K, vec, rot->perm + static_cast<size_t>(g) * rot->K,
                                                    rot->vec2 + static_cast<size_t>(g) * rot->K, 0, codes, scales,
                                                    static_cast<cudaStream_t>(stream));
-    return e2 == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+    return finish(e2 == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA, stream);
   }
   if (rotate_quantize_prefers_team(M, rot->K))
-    return launch_rotate_quantize_team(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream));
+    return finish(launch_rotate_quantize_team(X_bf16, ldx, M, rot->K, vec, codes, scales, static_cast<cudaStream_t>(stream)), stream);
   const cudaError_t e = launch_rotate_quantize(X_bf16, ldx, M, rot->K, vec, 0, codes, scales, static_cast<cudaStream_t>(stream));
-  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return finish(e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA, stream);
 }
 
 trdq_status trdq_norm_rotate_quantize(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M,
@@ -526,7 +544,7 @@ trdq_status trdq_norm_rotate_quantize(const trdq_rotation* rot, int32_t t, const
   if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const cudaError_t e = launch_norm_rotate_quantize(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, shift_bf16,
                                                     scale_bf16, rows_per_sample, eps, codes, scales, static_cast<cudaStream_t>(stream));
-  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return finish(e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA, stream);
 }
 
 static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t* const codes[2], const float* const scales[2],
@@ -547,8 +565,8 @@ static trdq_status linear_common(const trdq_weights* w, int32_t t, const int8_t*
   if (M[0] == 0 && M[1] == 0) return TRDQ_OK;
   if (check_bias(bias) != TRDQ_OK) return TRDQ_ERR_ALIGN;
   if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
-  if (w->wbits == 8) return launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream), act);
-  return launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream), act);
+  if (w->wbits == 8) return finish(launch_gemm_w8(w, g, seg, bias, raw, static_cast<cudaStream_t>(stream), act), stream);
+  return finish(launch_gemm_w4(w, g, seg, bias, static_cast<cudaStream_t>(stream), act), stream);
 }
 
 trdq_status trdq_linear(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M, const void* bias_bf16,
@@ -602,7 +620,7 @@ trdq_status trdq_linear_splitk(const trdq_weights* w, int32_t t, const int8_t* c
   if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   if (workspace_bytes < static_cast<uint64_t>(splits) * static_cast<uint64_t>(M) * static_cast<uint64_t>(w->N) * 4u) return TRDQ_ERR_NOMEM;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
-  return launch_gemm_w8_splitk(w, g, seg, bias_bf16, splits, static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream));
+  return finish(launch_gemm_w8_splitk(w, g, seg, bias_bf16, splits, static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream)), stream);
 }
 
 trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const int8_t* codes, const float* scales, int32_t M,
@@ -618,7 +636,7 @@ trdq_status trdq_linear_splitk_static(const trdq_weights* w, int32_t t, const in
   if (check_bias(bias_bf16) != TRDQ_OK) return TRDQ_ERR_ALIGN;
   if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   const GemmSegment seg{codes, scales, Y_bf16, ldy, M};
-  return launch_gemm_w8_splitk_static(w, g, seg, bias_bf16, splits, static_cast<cudaStream_t>(stream));
+  return finish(launch_gemm_w8_splitk_static(w, g, seg, bias_bf16, splits, static_cast<cudaStream_t>(stream)), stream);
 }
 
 trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const void* X_bf16, int64_t ldx, int32_t M, uint8_t* codes,
@@ -637,7 +655,7 @@ trdq_status trdq_rotate_quantize_asym(const trdq_rotation* rot, int32_t t, const
   if (!on_current_device(rot->device)) return TRDQ_ERR_MISMATCH;
   const cudaError_t e = launch_rotate_quantize_asym(X_bf16, ldx, M, rot->K, rot->act_vec + static_cast<size_t>(g) * rot->K, codes, scales,
                                                     zero_points, static_cast<cudaStream_t>(stream));
-  return e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return finish(e == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA, stream);
 }
 
 trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* codes, const float* scales, const int32_t* zero_points,
@@ -655,7 +673,7 @@ trdq_status trdq_linear_asym(const trdq_weights* w, int32_t t, const uint8_t* co
   if (!on_current_device(w->device)) return TRDQ_ERR_MISMATCH;
   GemmSegment seg[2] = {GemmSegment{reinterpret_cast<const int8_t*>(codes), scales, Y_bf16, ldy, M}, GemmSegment{nullptr, nullptr, nullptr, ldy, 0}};
   const int32_t* zp[2] = {zero_points, nullptr};
-  return launch_gemm_w8_asym(w, g, seg, zp, bias_bf16, static_cast<cudaStream_t>(stream));
+  return finish(launch_gemm_w8_asym(w, g, seg, zp, bias_bf16, static_cast<cudaStream_t>(stream)), stream);
 }
 
 trdq_status trdq_gemm_i32(const trdq_weights* w, int32_t t, const int8_t* codes, int32_t M, int32_t* acc, int64_t ldacc, void* stream) {
@@ -723,7 +741,7 @@ trdq_status trdq_selftest_wait_expiry(void* stream) {
   uint32_t* status = device_status_word();
   if (!status) return TRDQ_ERR_CUDA;
   selftest_wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status);
-  return cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA;
+  return finish(cudaGetLastError() == cudaSuccess ? TRDQ_OK : TRDQ_ERR_CUDA, stream);
 }
 
 trdq_status trdq_device_status(uint32_t* word) {

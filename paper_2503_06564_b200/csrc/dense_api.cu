@@ -170,7 +170,8 @@ trdq_status trdq_rotate_dense_quantize(const trdq_rotation* rot, int32_t t, cons
   const auto misaligned = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
   if (ldx % 8 != 0 || misaligned(X_bf16, 16) || misaligned(codes, 16) || misaligned(scales, 4) || misaligned(workspace, 4)) return TRDQ_ERR_ALIGN;
   if (workspace_bytes < rotate_dense_workspace_bytes(M, rot->K)) return TRDQ_ERR_NOMEM;
-  return launch_rotate_dense_quantize(rot, g, X_bf16, ldx, M, codes, scales, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream));
+  return trdq::finish(launch_rotate_dense_quantize(rot, g, X_bf16, ldx, M, codes, scales, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream)),
+                      stream);
 }
 
 // Eq. 6-7 for one block, on the host in double.  Step k: d = column of the largest |Y| (Y = X R^1 .. R^(k-1), first

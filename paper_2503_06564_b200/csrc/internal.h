@@ -68,6 +68,9 @@ struct PerDevice {
 };
 using PerDeviceFlag = PerDevice<bool>;
 
+// TRDQ_DEBUG=1: waits for the call's own work and turns a device error or an expired wait into the call's return code.
+trdq_status finish(trdq_status st, void* stream);
+
 uint32_t* device_status_word();  // device address of the status word of the current device (nullptr on failure)
 
 // rotate_quantize.cu

@@ -523,3 +523,29 @@ def test_kernel_choice_and_tensor_pipe_ceiling():
     per_cluster = 16384 * 2 * 256 * 256 * 32
     assert ops % per_cluster == 0 and 1 <= ops // per_cluster <= sms // 2
     assert 1000.0 < tops < 6000.0, tops           # the tensor pipe alone: a few PTOPS on this part
+
+
+def test_debug_mode_reports_at_the_call():
+    """TRDQ_DEBUG=1 (read once per process, hence a child process): every online call waits for its own work, so the
+    self-test's expired wait comes back from that very call, the word is cleared, and ordinary calls still return OK."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_2503_06564_b200 import trdq\n"
+        "lib = trdq.lib()\n"
+        "st = trdq._stream()\n"
+        "assert lib.trdq_selftest_wait_expiry(st) == 9\n"
+        "assert trdq.trdq_device_status() == 0\n"
+        "rot = trdq.Rotation(1152, [0, 1000], np.ones((1, 1152), np.int8))\n"
+        "x = torch.randn((3000, 1152), device='cuda').to(torch.bfloat16)\n"
+        "w = trdq.trdq_prepare_weights(rot, (torch.randn((256, 1152), device='cuda') * 0.02).to(torch.bfloat16), 8)\n"
+        "c, s = trdq.trdq_rotate_quantize(rot, 0, x)\n"
+        "y = trdq.trdq_linear(w, 0, c, s, None)\n"
+        "assert torch.isfinite(y.float()).all().item() and trdq.trdq_device_status() == 0\n"
+        "print('debug ok')\n")
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, TRDQ_DEBUG="1"), capture_output=True, text=True,
+                         timeout=600)
+    assert res.returncode == 0 and "debug ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
