@@ -15,6 +15,7 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "lane_group.cuh"
 #include "ptx.cuh"
 
 namespace trdq {
@@ -22,7 +23,6 @@ namespace {
 
 constexpr int kMaxWarps = 12;        // 12 x 32 threads x <= 168 registers fill the register file
 constexpr int kVecPadFloats = 4;     // the fused vector of block b starts at float b * (128 + 4): see the staging loop
-constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23
 
 struct alignas(64) TeamParams {
   // Both maps view a row as K/64 (K/128) column boxes: dims (column in box, row, box), so that ONE copy moves a tile of R
@@ -43,12 +43,6 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
-}
-
-__device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
-  const uint32_t lo = __byte_perm(__float_as_uint(a.x), __float_as_uint(a.y), 0x0040);
-  const uint32_t hi = __byte_perm(__float_as_uint(b.x), __float_as_uint(b.y), 0x0040);
-  return __byte_perm(lo, hi, 0x5410);
 }
 
 // max(|a|, |b|, |c|) in one instruction

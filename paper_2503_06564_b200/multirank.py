@@ -10,6 +10,8 @@ import os
 import socket
 import subprocess
 import sys
+import tempfile
+import time
 from typing import List, Optional, Sequence, Tuple
 
 
@@ -66,22 +68,34 @@ def spawn_ranks(world: int, argv: Sequence[str], timeout: Optional[float] = None
     if world < 1:
         raise ValueError("world size must be positive")
     port = free_port()
+    out_file = tempfile.TemporaryFile(mode="w+")
     procs: List[subprocess.Popen] = []
     for rank in range(world):
         procs.append(subprocess.Popen(list(argv), env=rank_environment(rank, world, port),
-                                      stdout=subprocess.PIPE if rank == 0 else sys.stderr, text=rank == 0))
+                                      stdout=out_file if rank == 0 else sys.stderr))
+    # Rank 0's output goes to a temporary file (no pipe to fill up); all children are polled, and the first failure or the
+    # deadline ends the others, so that a rank lost before a collective cannot leave the rest waiting for ever.
     worst, out0 = 0, ""
+    deadline = None if timeout is None else time.monotonic() + timeout
     try:
-        out0, _ = procs[0].communicate(timeout=timeout)
-        worst = procs[0].returncode
-        for p in procs[1:]:
-            rc = p.wait(timeout=timeout)
-            worst = worst or rc
-    except subprocess.TimeoutExpired:
-        worst = 124
+        while True:
+            codes = [p.poll() for p in procs]
+            failed = [c for c in codes if c not in (None, 0)]
+            if failed:
+                worst = failed[0]
+                break
+            if all(c == 0 for c in codes):
+                break
+            if deadline is not None and time.monotonic() > deadline:
+                worst = 124
+                break
+            time.sleep(0.05)
     finally:
         for p in procs:
             if p.poll() is None:
                 p.kill()
                 p.wait()
+        out_file.seek(0)
+        out0 = out_file.read()
+        out_file.close()
     return worst, out0

@@ -96,5 +96,12 @@ def test_spawn_ranks_gives_every_rank_its_environment(tmp_path):
     bad.write_text("import os, sys\nsys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
     rc, _ = multirank.spawn_ranks(2, [sys.executable, str(bad)], timeout=60)
     assert rc == 3
+    # a rank that never finishes is ended when another one fails (no waiting for a collective that cannot complete)
+    hang = tmp_path / "hang.py"
+    hang.write_text("import os, sys, time\nif os.environ['RANK'] == '0': time.sleep(600)\nsys.exit(5)\n")
+    import time
+    t0 = time.monotonic()
+    rc, _ = multirank.spawn_ranks(2, [sys.executable, str(hang)], timeout=120)
+    assert rc == 5 and time.monotonic() - t0 < 60
     with pytest.raises(ValueError):
         multirank.spawn_ranks(0, [sys.executable, str(bad)])
