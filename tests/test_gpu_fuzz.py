@@ -1,5 +1,7 @@
 """Seeded random shapes through the whole path (rotate + quantize, both GEMM kernels, 8- and 4-bit weights,
 with and without smoothing and bias) against the oracle: small problems, many corner combinations."""
+import os
+
 import numpy as np
 import pytest
 
@@ -8,6 +10,7 @@ from paper_2503_06564_b200 import workloads as WL
 from tests.util import bf16_to_f32_np, check_output, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
+LARGE_SEEDS = int(os.environ.get("TRDQ_FUZZ_SEEDS", "10"))   # more seeds for a soak run
 
 
 @pytest.mark.parametrize("seed", list(range(12)))
@@ -56,6 +59,34 @@ def test_random_problem(seed):
     assert np.array_equal(wq_dev.cpu().numpy(), qw_ref if wbits == 8 else pk_ref)
     l2, ulps = check_output(bf16_to_f32_np(y), y_ref, max_ulp=2.0, rel_l2=2e-3)
     assert ulps <= 1.0
+    assert trdq.trdq_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", list(range(LARGE_SEEDS)))
+def test_random_large_rotate_quantize(seed):
+    """Row counts in the thousands with random row widths (1 to 80 blocks), row strides and group vectors: the shapes that
+    go to the one-thread-per-block team kernel with every team size it has, ragged last tiles included."""
+    import torch
+    from paper_2503_06564_b200 import trdq
+    rng = np.random.default_rng(5000 + seed)
+    nb = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 11, 16, 18, 24, 32, 33, 36, 40, 64, 72, 80]))
+    K = 128 * nb
+    M = int(rng.integers(150, max(151, min(30000, 24_000_000 // K))))
+    pad = int(rng.choice([0, 8, 64, 136]))
+    signs = (rng.integers(0, 2, (1, K)) * 2 - 1).astype(np.int8)
+    smooth = rng.uniform(0.3, 3.0, (1, K)).astype(np.float32) if rng.integers(0, 2) else None
+    rot = trdq.Rotation(K, [0, 1000], signs, smooth)
+    x = rng.standard_normal((M, K)).astype(np.float32) * np.float32(rng.uniform(0.1, 5.0))
+    x[:, rng.choice(K, max(1, K // 64), replace=False)] *= 25.0
+    x[rng.integers(0, M)] = 0.0
+    xb = WL.to_bf16_bits(x.astype(np.float64))
+    wide = torch.zeros((M, K + pad), dtype=torch.bfloat16, device="cuda")
+    wide[:, :K] = to_dev_bf16(xb)
+    codes, scales = trdq.trdq_rotate_quantize(rot, 0, wide[:, :K])
+    act, _ = O.fused_vectors(signs[0], None if smooth is None else smooth[0])
+    q_ref, s_ref = O.rotate_quantize(xb, act)
+    assert np.array_equal(scales.cpu().numpy(), s_ref), (M, K, pad, trdq.trdq_kernel_choice(0, M, K))
+    assert np.array_equal(codes.cpu().numpy(), q_ref), (M, K, pad, trdq.trdq_kernel_choice(0, M, K))
     assert trdq.trdq_device_status() == 0
 
 
