@@ -428,8 +428,9 @@ int max_clusters(int dev) {
 
 // Tile width: waves of resident clusters times the time of one tile.  The kernel is bound by operand delivery from L2,
 // so a tile costs what it loads, (256 + BN) panel rows of K bytes; wider tiles load less per multiply-add.  Checked
-// against a sweep of all three widths over the layer shapes at M = 4096 ... 32768: the model picks the fastest width or
-// one within 2 % of it (the earlier model, waves x (BN + 24), left 4 - 15 % on the table at M >= 16384).
+// against a sweep of all three widths over the layer shapes at M = 4096 ... 32768 with the banded tile order: the model
+// picks the fastest width or one within 2 % of it (the earlier model, waves x (BN + 24), left 4 - 15 % on the table at
+// M >= 16384; without the ragged-tile factor N = 1152 got width 256 where 192 is 2 - 3 % faster).
 // Returns the index into kTileN (and the resident clusters of that width), or -1 if the kernel cannot run here.
 int pair_tile_choice(int64_t tiles_m, int N, int dev, int* clusters_out) {
   int best = -1;
@@ -439,9 +440,13 @@ int pair_tile_choice(int64_t tiles_m, int N, int dev, int* clusters_out) {
     const int bn = kTileN[i];
     clusters_of[i] = bn == 128 ? max_clusters<128>(dev) : bn == 192 ? max_clusters<192>(dev) : max_clusters<256>(dev);
     if (clusters_of[i] <= 0) continue;
-    const int64_t tiles = tiles_m * ((N + bn - 1) / bn);
-    const int64_t waves = (tiles + clusters_of[i] - 1) / clusters_of[i];
-    const double cost = static_cast<double>(waves) * (256.0 + bn);
+    const int64_t tiles_n = (N + bn - 1) / bn;
+    const int64_t tiles = tiles_m * tiles_n;
+    // whole waves while there are few of them; with four or more the persistent clusters even a partial wave out
+    const double waves = tiles >= 4ll * clusters_of[i] ? static_cast<double>(tiles) / clusters_of[i]
+                                                       : static_cast<double>((tiles + clusters_of[i] - 1) / clusters_of[i]);
+    // a ragged last column tile loads and multiplies columns that do not exist (N = 1152 in tiles of 256: 11 %)
+    const double cost = waves * (256.0 + bn) * (static_cast<double>(tiles_n * bn) / N);
     if (cost < best_cost) {
       best_cost = cost;
       best = i;
