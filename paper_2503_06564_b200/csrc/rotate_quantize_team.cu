@@ -107,14 +107,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) rotate_quantize_team_kernel
   const int num_tiles = (p.M + R - 1) / R;
   const int stride = gridDim.x * p.teams;
   const int first = team * gridDim.x + blockIdx.x;
-  if (tt == 0) {
-    for (int s = 0; s < 2; ++s) {
-      const int tile = first + s * stride;
-      if (tile < num_tiles) {
-        mbar_arrive_expect_tx(bar_full + 8 * s, in_bytes);
-        tma_load_3d(team_base + s * in_bytes, &p.tmap_x, 0, tile * R, 0, bar_full + 8 * s);  // all 2 * nb column boxes in one copy
-      }
-    }
+  // Only the FIRST tile of every team is requested here; the second one follows when the first has landed (below).  All
+  // teams of all CTAs start together, so asking for both at once doubles the burst every first tile has to wait behind.
+  if (tt == 0 && first < num_tiles) {
+    mbar_arrive_expect_tx(bar_full, in_bytes);
+    tma_load_3d(team_base, &p.tmap_x, 0, first * R, 0, bar_full);  // all 2 * nb column boxes in one copy
   }
 
   // consecutive threads = consecutive rows of one block column
@@ -133,6 +130,10 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) rotate_quantize_team_kernel
     if (tt < R) row_max[((it + 1) % 3) * R + tt] = 0u;
 
     w.wait(bar_full + 8 * s, phase);
+    if (it == 0 && tt == 0 && tile + stride < num_tiles) {  // the team's second tile, into the other stage
+      mbar_arrive_expect_tx(bar_full + 8, in_bytes);
+      tma_load_3d(team_base + in_bytes, &p.tmap_x, 0, (tile + stride) * R, 0, bar_full + 8);
+    }
     // v[32h + 4j + i] = elements (2i, 2i+1) of 16-byte chunk j of half h, times the fused vector
     float2 v[64];
 #pragma unroll
