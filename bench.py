@@ -230,6 +230,45 @@ class KernelPass:
             self.graph.replay()
         torch.cuda.synchronize()
 
+    @classmethod
+    def per_layer_us(cls, layers, wl, reps: int = 5):
+        """Microseconds per launch of each layer of a block, both kernel kinds: the launches of that layer over all blocks
+        (distinct buffers) replayed back to back from a graph."""
+        import torch
+        from paper_2503_06564_b200 import trdq
+        t = int(wl.timesteps()[0])
+        per_block = len(wl.layers + wl.extra_layers)
+        out = []
+        for j, layer in enumerate(wl.layers + wl.extra_layers):
+            entry = {"layer": layer.name}
+            for which in ("rq", "gemm"):
+                self = cls.__new__(cls)
+                sel = [(k, ws) for i, (k, ws) in enumerate(zip(layers._keep, layers._extra)) if i % per_block == j]
+
+                def issue():
+                    for (rot, w, x, codes, scales, bias, y), ws in sel:
+                        if which == "rq" and ws is not None:
+                            trdq.trdq_rotate_dense_quantize(rot, t, x, codes, scales, ws)
+                        elif which == "rq":
+                            trdq.trdq_rotate_quantize(rot, t, x, codes, scales)
+                        else:
+                            trdq.trdq_linear(w, t, codes, scales, bias, y)
+
+                self.graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(self.graph, capture_error_mode="thread_local"):
+                    issue()
+                ms, _ = self.ms(reps=reps)
+                us = ms * 1e3 / len(sel)
+                m = layer.M or wl.M
+                if which == "rq":
+                    entry["rotate_quantize_us"] = us
+                    entry["rotate_quantize_gbs"] = m * (3.0 * layer.K + 4.0) / (us * 1e-6) / 1e9
+                else:
+                    entry["linear_us"] = us
+                    entry["linear_tops"] = 2.0 * m * layer.N * layer.K / (us * 1e-6) / 1e12
+            out.append(entry)
+        return out
+
     def ms(self, reps: int = 0, min_seconds: float = 0.0):
         """(ms per pass, seconds timed): `reps` passes, or as many as fill `min_seconds`; a tenth of them untimed first."""
         once = time_region(lambda i: self.graph.replay(), 3) / 3
@@ -574,6 +613,13 @@ def run_ours(args, wl: WL.Workload):
     roof_gemm["brief"] = {k: burst_gemm[k] for k in ("achieved", "peak", "frac", "frac_nominal", "seconds_timed", "peak_source")}
     roof_rq["sustained"] = {k: rq_long[k] for k in ("achieved", "frac", "frac_nominal", "seconds_timed")}
     roof_rq["peak_source"] += " (best of ten 4 GB copies: a burst figure, compared with the brief pass)"
+    per_layer_clocks = None
+    if rank == 0:   # per-layer passes: microseconds per launch of every layer shape, in the state the long passes left the part in
+        sampler3 = ClockSampler(local_rank)
+        sampler3.start()
+        for entry, timing in zip(per_layer, KernelPass.per_layer_us(layers, wl, reps=10)):
+            entry.update({k: v for k, v in timing.items() if k != "layer"})
+        per_layer_clocks = sampler3.stop()
     ceiling = None
     if rank == 0 and wl.wbits == 8:
         c = microbench.mma_ceiling(65536, 5)
@@ -649,6 +695,9 @@ def run_ours(args, wl: WL.Workload):
         "roofline_rotate_quantize": roof_rq,
         "mma_ceiling": ceiling,
         "kernels_per_layer": per_layer,
+        "kernels_per_layer_note": "us per launch: that layer's launches over all blocks replayed from a graph, ten times, right after the "
+                                  "two-second passes (the part is still at its power-capped clocks)",
+        "kernels_per_layer_clocks": per_layer_clocks,
         "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps},
         "gpu_launches": (3 if dense else 2) * n_ops * args.steps,
