@@ -83,6 +83,54 @@ __device__ __forceinline__ uint32_t pack4(float2 a, float2 b) {
   return __byte_perm(lo, hi, 0x5410);
 }
 
+// The lane's four 16-byte chunks of bf16 values widened to fp32 pairs (exact: the 16 bits become the high half of the
+// fp32 pattern): v[4c + j] = elements (2j, 2j+1) of chunk c.
+__device__ __forceinline__ void widen_chunks_lanes4(const uint4 (&raw)[4], float2 (&v)[16]) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[4 * c + j] = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+  }
+}
+
+// The same, times the fused vector (sv points at the lane's first column; chunk c is 32 columns = 16 pairs further).
+__device__ __forceinline__ void scale_chunks_lanes4(const uint4 (&raw)[4], const float2* sv, float2 (&v)[16]) {
+  widen_chunks_lanes4(raw, v);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[4 * c + j] = __fmul2_rn(v[4 * c + j], sv[16 * c + j]);
+  }
+}
+
+// Largest magnitude of the block: the lane's 32 values, then the four lanes of the group.
+__device__ __forceinline__ float absmax_lanes4(const float2 (&v)[16]) {
+  float m = 0.0f;
+#pragma unroll
+  for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  return fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+}
+
+// Symmetric int8 codes of the lane's 32 values to dst (+ 32 c per chunk): q = rne(fl(v * inv)) with inv = fl(127 / amax).
+// The product must be rounded to fp32 before the magic addition rounds it to an integer.  A packed multiply feeding a
+// packed add gets contracted into one fused operation (a single rounding) by the assembler, so the product is written
+// as fma(v, inv, zero) with `zero` a kernel argument equal to 0.0f: one rounding of v * inv, nothing left to contract.
+__device__ __forceinline__ void quantize_store_lanes4(const float2 (&v)[16], float amax, float zero, int8_t* dst) {
+  const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+  const float2 inv2 = make_float2(inv, inv);
+  const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
+  const float2 zero2 = make_float2(zero, zero);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    float2 q[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
+    *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
+  }
+}
+
 // 128-point transform of one block spread over four lanes (16 fp32 pairs per lane, layout as described above).
 __device__ __forceinline__ void wht128_lanes4(float2 (&v)[16], int lane4) {
   // h = 1: inside a pair

@@ -88,12 +88,7 @@ norm_rotate_quantize_rows_kernel(const uint16_t* __restrict__ x, int64_t ldx, in
 
     // v[4c + j] = elements (2j, 2j+1) of chunk c
     float2 v[16];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) v[4 * c + j] = bf16x2_to_float2(w[j]);
-    }
+    widen_chunks_lanes4(raw, v);
     fetch(tile + gridDim.x);  // next tile's rows are in flight while this one is reduced and transformed
 
     // statistics of this group's 128 values: mean, then the sum of squared deviations from it
@@ -151,28 +146,13 @@ norm_rotate_quantize_rows_kernel(const uint16_t* __restrict__ x, int64_t ldx, in
 
     wht128_lanes4(v, lane4);
 
-    float m = 0.0f;
-#pragma unroll
-    for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    const float m = absmax_lanes4(v);
     if (valid && lane4 == 0) atomicMax(&row_max[buf][r], __float_as_uint(m));
     __syncthreads();
 
     if (valid) {
       const float amax = __uint_as_float(row_max[buf][r]);
-      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-      const float2 inv2 = make_float2(inv, inv);
-      const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
-      const float2 zero2 = make_float2(zero, zero);  // fma(v, inv, 0): the product rounded once, nothing for the assembler to contract
-      int8_t* dst = codes + static_cast<int64_t>(row) * K + col0;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float2 q[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
-        *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
-      }
+      quantize_store_lanes4(v, amax, zero, codes + static_cast<int64_t>(row) * K + col0);
       if (b == 0 && lane4 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
     }
   }

@@ -291,45 +291,18 @@ rotate_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, in
 
     // v[4c + j] = elements (2j, 2j+1) of chunk c, scaled by the fused vector
     float2 v[16];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 xv = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
-        v[4 * c + j] = __fmul2_rn(xv, sv[16 * c + j]);
-      }
-    }
+    scale_chunks_lanes4(raw, sv, v);
     fetch(tile + gridDim.x);  // next tile's rows are in flight while this one is transformed
 
     wht128_lanes4(v, lane4);
 
-    float m = 0.0f;
-#pragma unroll
-    for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    const float m = absmax_lanes4(v);
     if (valid && lane4 == 0) atomicMax(&row_max[buf][r], __float_as_uint(m));
     __syncthreads();
 
     if (valid) {
       const float amax = __uint_as_float(row_max[buf][r]);
-      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-      const float2 inv2 = make_float2(inv, inv);
-      const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
-      // The product must be rounded to fp32 before the magic addition rounds it to an integer.  A packed
-      // multiply feeding a packed add gets contracted into one fused operation (a single rounding) by
-      // the assembler, so the product is written as fma(v, inv, zero) with `zero` a kernel argument
-      // equal to 0.0f: one rounding of v * inv, and nothing left to contract.
-      const float2 zero2 = make_float2(zero, zero);
-      int8_t* dst = codes + row * K + col0;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float2 q[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
-        *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
-      }
+      quantize_store_lanes4(v, amax, zero, codes + row * K + col0);
       if (b == 0 && lane4 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
     }
   }
@@ -399,15 +372,7 @@ rotate2_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, i
     const bool valid = active && row < M;
 
     float2 v[16];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 xv = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
-        v[4 * c + j] = __fmul2_rn(xv, sv[16 * c + j]);
-      }
-    }
+    scale_chunks_lanes4(raw, sv, v);
     fetch(tile + gridDim.x);
     wht128_lanes4(v, lane4);  // first rotation
     if (active) {
@@ -431,28 +396,13 @@ rotate2_quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, i
     }
     wht128_lanes4(v, lane4);  // second rotation
 
-    float m = 0.0f;
-#pragma unroll
-    for (int p = 0; p < 16; ++p) m = fmaxf(fmaxf(m, fabsf(v[p].x)), fabsf(v[p].y));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    const float m = absmax_lanes4(v);
     if (valid && lane4 == 0) atomicMax(&row_max[buf][r], __float_as_uint(m));
     __syncthreads();  // row maxima complete; all gathers done, the row buffer may be overwritten
 
     if (valid) {
       const float amax = __uint_as_float(row_max[buf][r]);
-      const float inv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-      const float2 inv2 = make_float2(inv, inv);
-      const float2 magic2 = make_float2(kRoundMagic, kRoundMagic);
-      const float2 zero2 = make_float2(zero, zero);  // see rotate_quantize_rows_kernel: keeps the product separately rounded
-      int8_t* dst = codes + row * K + col0;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float2 q[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) q[j] = __fadd2_rn(__ffma2_rn(v[4 * c + j], inv2, zero2), magic2);
-        *reinterpret_cast<uint2*>(dst + 32 * c) = make_uint2(pack4(q[0], q[1]), pack4(q[2], q[3]));
-      }
+      quantize_store_lanes4(v, amax, zero, codes + row * K + col0);
       if (b == 0 && lane4 == 0) scales[row] = __fdiv_rn(amax, 127.0f);
     }
   }
@@ -509,14 +459,10 @@ rotate_quantize_rows_asym_kernel(const __nv_bfloat16* __restrict__ x, int64_t ld
     float2 v[16];
     if (valid) {
       const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx + col0);
+      uint4 raw[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint4 raw = __ldg(src + 4 * c);
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          v[4 * c + j] = __fmul2_rn(make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u)), sv[16 * c + j]);
-      }
+      for (int c = 0; c < 4; ++c) raw[c] = __ldg(src + 4 * c);
+      scale_chunks_lanes4(raw, sv, v);
     } else {
 #pragma unroll
       for (int p = 0; p < 16; ++p) v[p] = make_float2(0.0f, 0.0f);
